@@ -1,0 +1,221 @@
+/*
+ * csd.h - C ABI of the review-step library for Cascade Speculative Drafting (arXiv 2312.11462).
+ *
+ * The library is hand-written CUDA for sm_100a.  It never allocates device memory: every device
+ * buffer (weights, KV cache and activations inside a workspace, logits, token buffers) is
+ * allocated by the caller and passed in as a plain pointer.  Handles (csd_model, csd_mag) are
+ * small host objects owned by the library and released by the matching *_destroy call.
+ *
+ * Conventions
+ *   - A pointer named *_dev is device memory, *_host is host memory.  Device buffers must stay
+ *     valid until the stream has passed the call.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  All calls except
+ *     csd_cascade_generate and csd_device_status only enqueue work; argument and shape errors
+ *     are returned synchronously and nothing is enqueued in that case.
+ *   - Errors found on the device (token id outside [0, vocab), a probe limit reached) never trap:
+ *     the kernel records a code in a status word, substitutes a safe value and carries on;
+ *     csd_device_status waits for the stream and returns-and-clears that word.
+ *   - No call falls back to the CPU.  Without a CUDA device every compute call returns
+ *     CSD_ERR_CUDA.
+ */
+#ifndef CSD_H
+#define CSD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    CSD_OK = 0,
+    CSD_ERR_INVALID_ARG = 1, /* null pointer, negative size, value out of its documented range */
+    CSD_ERR_SHAPE = 2,       /* a model dimension the kernels do not support                    */
+    CSD_ERR_CAPACITY = 3,    /* kv_len + m > max_seq, workspace too small, block too long        */
+    CSD_ERR_OOM = 4,         /* host allocation of a handle failed                              */
+    CSD_ERR_CUDA = 5,        /* a CUDA runtime call failed (see csd_last_cuda_error)            */
+    CSD_ERR_BAD_TOKEN = 6,   /* device status: a token id was outside [0, vocab)                */
+    CSD_ERR_TIMEOUT = 7,     /* device status: a bounded probe loop reached its limit           */
+    CSD_ERR_UNSUPPORTED = 8
+} csd_status;
+
+const char* csd_status_string(csd_status s);
+/* Text of the last CUDA runtime error seen by this thread's calls ("" if none). */
+const char* csd_last_cuda_error(void);
+/* Waits for `stream`, stores the device status word (a csd_status) in *code_out, clears it. */
+csd_status csd_device_status(void* stream, int* code_out);
+
+/* ---------------------------------------------------------------------------------------------
+ * Models.  The paper names the model families only (Section 5.1: a LLaMA-family 7B target with
+ * a 68M draft; FLAN-T5 xxl with base and small drafts), so the architecture constants are the
+ * public ones of those families:
+ *   arch 0  decoder-only: pre-norm RMSNorm, rotary embedding on head-dim halves (i, i+Dh/2),
+ *           scores scaled by 1/sqrt(Dh), SwiGLU feed-forward, untied output head, no biases.
+ *   arch 1  encoder-decoder: RMS norm without mean-centring, unscaled scores plus a bucketed
+ *           relative-position bias shared by all layers of a stack (bidirectional buckets in
+ *           the encoder, causal in the decoder), cross-attention, gated-GELU (tanh form)
+ *           feed-forward, untied output head, no biases.
+ * Arithmetic: bf16 weights, fp32 activations and accumulation, K/V rounded to bf16
+ * (nearest-even) when a position is appended to the cache.
+ *
+ * Weight blob (device, bf16, every tensor [out, in] row-major and starting on a 256-byte
+ * boundary), in this order:
+ *   embed [vocab, d_model]
+ *   arch 1 only: enc_rel_bias [rel_buckets, n_heads];
+ *                per encoder layer { norm1 [d], wq, wk, wv [d_inner, d], wo [d, d_inner],
+ *                                    norm2 [d], wgate, wup [d_ff, d], wdown [d, d_ff] };
+ *                enc_final_norm [d]; dec_rel_bias [rel_buckets, n_heads]
+ *   per decoder layer { norm1, wq, wk, wv, wo,
+ *                       arch 1 only: norm_x, xq, xk, xv, xo (cross-attention),
+ *                       norm2, wgate, wup, wdown }
+ *   final_norm [d]; lm_head [vocab, d_model]
+ * with d_inner = n_heads * d_head.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct csd_model csd_model;
+
+typedef struct {
+    int32_t arch;         /* 0 decoder-only, 1 encoder-decoder                              */
+    int32_t n_layers;     /* decoder layers                                                  */
+    int32_t n_enc_layers; /* encoder layers (arch 1)                                         */
+    int32_t d_model;      /* multiple of 8                                                   */
+    int32_t n_heads;
+    int32_t d_head;       /* 32, 64 or 128                                                   */
+    int32_t d_ff;         /* multiple of 8                                                   */
+    int32_t vocab;
+    int32_t max_seq;      /* decoder KV capacity in positions                                */
+    int32_t max_rows;     /* most rows one review forward takes, <= 17                       */
+    int32_t max_enc_len;  /* arch 1: most encoder positions                                  */
+    int32_t rel_buckets;  /* arch 1: relative-position buckets (32)                          */
+    int32_t rel_max_dist; /* arch 1: distance at which buckets saturate (128)                */
+    float norm_eps;
+    float rope_theta;     /* arch 0                                                          */
+} csd_model_config;
+
+#define CSD_MAX_ROWS 17
+
+size_t csd_model_weight_bytes(const csd_model_config* cfg);
+/* Workspace = KV cache (+ cross-attention K/V), activations, split partials, tables. */
+size_t csd_model_workspace_bytes(const csd_model_config* cfg);
+
+/* Binds a model to caller-owned weights and workspace (both device, 256-byte aligned, at least
+ * the sizes above; the caller keeps them alive until csd_model_destroy).  Enqueues the
+ * one-off table set-up (rotary cos/sin, relative-position bias by distance) on `stream`. */
+csd_status csd_model_create(const csd_model_config* cfg, const void* weights_bf16_dev, size_t weight_bytes,
+                            void* workspace_dev, size_t workspace_bytes, void* stream, csd_model** out);
+csd_status csd_model_destroy(csd_model* m);
+
+/* arch 1: runs the encoder over n tokens (1 <= n <= max_enc_len) and fills the static
+ * cross-attention K/V of every decoder layer.  Must precede csd_review_forward. */
+csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int n, void* stream);
+
+/* The review forward: "reviewed by a target model in parallel ... in one single run" (Sections
+ * 1-2).  One pass over m rows (1 <= m <= max_rows) at positions kv_len .. kv_len+m-1: reads cache
+ * rows [0, kv_len), OVERWRITES rows [kv_len, kv_len+m), writes logits_out_dev [m, vocab] fp32
+ * row-major; row r is the model's next-token law after position kv_len+r, causal inside the
+ * block.  The caller commits accepted positions by passing a larger kv_len next time; rejected
+ * rows are simply overwritten (rollback is free). */
+csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
+                              float* logits_out_dev, void* stream);
+
+/* Y[m, N] = X[m, K] . W[N, K]^T, the weight-streaming contraction every layer of the review
+ * forward is made of (W bf16 row-major, X and Y fp32 row-major, fp32 accumulation).  Exposed
+ * for kernel-level tests and roofline measurements.  1 <= m <= 17, K multiple of 8. */
+size_t csd_linear_workspace_bytes(int m, int N, int K);
+csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, int m, float* Y_dev,
+                      void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Review rule (Section 2 "reviewing stage"; Section 3.1 for lenience and the greedy variant).
+ * For each of `rows` independent rows: drafted tokens x_1..x_k with draft laws q_i and target
+ * laws p_i = softmax(target_logits[i] / T):
+ *   temperature > 0: x_i is accepted iff u_i * q_i(x_i) < lenience * p_i(x_i) with u_i uniform
+ *     in [0,1); at the first rejection i the output token is drawn from norm(max(0, p_i - q_i))
+ *     (from p_i if that is empty); if all k are accepted it is drawn from p_{k+1}.
+ *   temperature == 0: greedy review: x_i is accepted iff it is the argmax of target_logits[i]
+ *     (ties: smallest index); the output token is the argmax at the first mismatch (or at k).
+ * q_i is softmax(draft_logits[i] / T), or the point mass on x_i where draft_logits_dev is NULL
+ * or onehot_dev[row, i] != 0 (statistical drafter).
+ * Uniforms: Philox4x32-10 with key (seed lo, seed hi) and counter (i, row, step lo, step hi);
+ * word 0 -> u_i, word 1 -> the resampling uniform of position i; u = (word >> 8) * 2^-24.  The
+ * resample is the inverse CDF in vocabulary order (smallest j with cumulative mass > u * total),
+ * evaluated in fp64.
+ * Layouts: target_logits_dev [rows, k+1, V] fp32, draft_logits_dev [rows, k, V] fp32 or NULL,
+ * onehot_dev [rows, k] int32 or NULL, draft_tokens_dev [rows, k] int32; outputs n_accepted_dev
+ * [rows], out_token_dev [rows] int32.  0 <= k <= 64.  A token id outside [0, V) is treated as
+ * rejected and sets the device status.
+ * ------------------------------------------------------------------------------------------- */
+size_t csd_spec_accept_workspace_bytes(int rows, int k, int V);
+csd_status csd_spec_accept(const float* target_logits_dev, const float* draft_logits_dev,
+                           const int32_t* onehot_dev, const int32_t* draft_tokens_dev, int rows, int k, int V,
+                           float temperature, float lenience, uint64_t seed, uint64_t step,
+                           int32_t* n_accepted_dev, int32_t* out_token_dev, void* workspace_dev,
+                           size_t workspace_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Max-Gram statistical drafter (Section 3.3, Appendix A): the longest suffix of the sequence
+ * (at most max_order tokens) that occurs in the haystack followed by at least one haystack
+ * token, earliest occurrence; the proposal is the haystack tokens after it.  When the haystack
+ * ends, or nothing matches (then one token comes from bigram_next[last token]), the search is
+ * repeated on the extended sequence until n tokens exist.  Lookup goes through a hash table of
+ * all n-grams of orders 1..max_order built once per haystack (exact under collisions: a slot
+ * is verified against the haystack).
+ * ------------------------------------------------------------------------------------------- */
+typedef struct csd_mag csd_mag;
+#define CSD_MAG_MAX_ORDER 32
+size_t csd_mag_workspace_bytes(int L, int max_order, int table_slots);
+/* haystack_dev [L] and bigram_next_dev [V] stay owned by the caller and must outlive the handle.
+ * table_slots: 0 = default (power of two >= 2 * L * max_order), else a power of two >= the
+ * number of n-grams (tests use small tables to force collisions). */
+csd_status csd_mag_create(const int32_t* haystack_dev, int L, int V, const int32_t* bigram_next_dev,
+                          int max_order, int table_slots, void* workspace_dev, size_t workspace_bytes,
+                          void* stream, csd_mag** out);
+csd_status csd_mag_destroy(csd_mag* g);
+/* seq_dev [T] (T >= 1), 1 <= n <= 64; writes out_tokens_dev [n] (may alias seq_dev + T). */
+csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32_t* out_tokens_dev,
+                         void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Algorithm 1 (CascadeSpeculativeDraftingStep) driven until max_new tokens exist.
+ * models[0] is the target, models[1 .. n_levels-1] the neural drafts, largest first; Max-Gram
+ * sits below them.  K is n_levels x n_levels, row-major, upper-triangular: K[r][c] is the budget
+ * of the slot that level c+1 drafts when level r reviews (level n_levels = Max-Gram, which
+ * proposes the slot's remaining budget in one call).  The for-loop over c is the horizontal
+ * cascade, the recursion into level c+1 the vertical cascade.  A review takes at most max_block
+ * drafted tokens (surplus drafts are dropped, which keeps the output law).  Lenience applies
+ * when a draft reviews, never when the target does.  Each level forwards every token it has not
+ * cached yet, in chunks of at most max_block+1 rows (this also serves as prompt prefill).
+ * Decoder-only models: haystack = prompt, init_seq = prompt.  Encoder-decoder: haystack =
+ * encoder input (the encoders are run here), init_seq = decoder start token(s).
+ * Host in, host out; the call returns after the stream has finished.
+ * ------------------------------------------------------------------------------------------- */
+typedef struct {
+    int64_t tokens;      /* tokens generated                                           */
+    int64_t reviews[8];  /* review calls per level (0 = target)                        */
+    int64_t forwards[8]; /* forward passes per level, catch-up chunks included        */
+    int64_t drafted[8];  /* drafted tokens presented to the level's reviews            */
+    int64_t accepted[8]; /* of which accepted                                          */
+    int64_t mag_calls;
+    int64_t mag_tokens;
+    int64_t kernel_launches; /* kernels this call enqueued                             */
+    double prefill_ms;   /* device time until the first target review starts (events)  */
+    double decode_ms;    /* device time from there to the last token (events)          */
+    double total_ms;     /* host wall time of the whole call, copies included          */
+} csd_cascade_stats;
+
+size_t csd_cascade_workspace_bytes(int vocab, int max_block, int seq_capacity, int haystack_len, int max_order);
+csd_status csd_cascade_generate(csd_model* const* models, int n_levels, const int32_t* K, int max_block,
+                                float lenience, float temperature, uint64_t seed, int max_order,
+                                const int32_t* haystack_host, int haystack_len,
+                                const int32_t* bigram_next_dev, const int32_t* init_seq_host, int init_len,
+                                int max_new, int32_t* out_tokens_host, int32_t* out_len,
+                                csd_cascade_stats* stats,
+                                void* workspace_dev, size_t workspace_bytes, void* stream);
+
+/* Host helper, exposed for tests: relative-position bucket of arch 1 (rel = key - query). */
+int csd_rel_bucket(int rel, int bidirectional, int n_buckets, int max_dist);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CSD_H */

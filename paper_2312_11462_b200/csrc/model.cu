@@ -1,0 +1,423 @@
+// Model handle and the review forward: one pass of a transformer over a block of m <= 17 rows
+// that streams the bf16 weights once, reads the bf16 K/V cache and appends the block to it.
+#include "model.cuh"
+#include <math.h>
+#include <new>
+#include <stdlib.h>
+#include <vector>
+
+namespace csd {
+
+// ---------------------------------------------------------------------------------------------
+// small kernels
+// ---------------------------------------------------------------------------------------------
+__global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E, int V, int d,
+                             float* __restrict__ x, int* status) {
+    const int r = blockIdx.x;
+    int t = tokens[r];
+    if (t < 0 || t >= V) {
+        if (threadIdx.x == 0) set_status(status, CSD_ERR_BAD_TOKEN);
+        t = 0;
+    }
+    const __nv_bfloat16* e = E + (size_t)t * d;
+    for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = __bfloat162float(e[i]);
+}
+
+// cos/sin of pos * theta^(-2i/Dh), evaluated in double once per model
+__global__ void rope_table_kernel(float* __restrict__ cs, float* __restrict__ sn, int max_seq, int half, double theta) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= max_seq * half) return;
+    const int pos = idx / half, i = idx % half;
+    const double ang = (double)pos * pow(theta, -(double)i / (double)half);
+    cs[idx] = (float)cos(ang);
+    sn[idx] = (float)sin(ang);
+}
+
+// bias_by_distance[h][i] = rel_bias[bucket[i]][h]
+__global__ void bias_table_kernel(const __nv_bfloat16* __restrict__ rel_bias, const int* __restrict__ bucket, int len,
+                                  int H, float* __restrict__ table) {
+    const int idx = blockIdx.x * blockDim.x + threadIdx.x;
+    if (idx >= len * H) return;
+    const int h = idx / len, i = idx % len;
+    table[idx] = __bfloat162float(rel_bias[(size_t)bucket[i] * H + h]);
+}
+
+// Rotates q (in place) and k of the block's rows, then appends k and v to the cache as bf16.
+// grid = (rows, heads); src is the fused projection output [rows, ld] with q|k|v column blocks.
+__global__ void rope_append_kernel(float* __restrict__ src, int ld, int q_off, int k_off, int v_off, int Dh,
+                                   int pos0, int cap, const float* __restrict__ cs, const float* __restrict__ sn,
+                                   __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc) {
+    const int r = blockIdx.x, h = blockIdx.y, pos = pos0 + r, half = Dh / 2;
+    float* row = src + (size_t)r * ld;
+    __nv_bfloat16* kdst = Kc + ((size_t)h * cap + pos) * Dh;
+    __nv_bfloat16* vdst = Vc + ((size_t)h * cap + pos) * Dh;
+    for (int i = threadIdx.x; i < half; i += blockDim.x) {
+        float k0 = row[k_off + h * Dh + i], k1 = row[k_off + h * Dh + i + half];
+        if (cs) {
+            const float c = cs[(size_t)pos * half + i], s = sn[(size_t)pos * half + i];
+            if (q_off >= 0) {
+                float* q = row + q_off + h * Dh;
+                const float q0 = q[i], q1 = q[i + half];
+                q[i] = q0 * c - q1 * s;
+                q[i + half] = q0 * s + q1 * c;
+            }
+            const float a = k0 * c - k1 * s, b = k0 * s + k1 * c;
+            k0 = a; k1 = b;
+        }
+        kdst[i] = __float2bfloat16_rn(k0);
+        kdst[i + half] = __float2bfloat16_rn(k1);
+        vdst[i] = __float2bfloat16_rn(row[v_off + h * Dh + i]);
+        vdst[i + half] = __float2bfloat16_rn(row[v_off + h * Dh + i + half]);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// layout helpers
+// ---------------------------------------------------------------------------------------------
+static size_t al128(size_t n) { return (n + 127) / 128 * 128; }
+
+struct BlobWalk {
+    const __nv_bfloat16* base;
+    size_t off = 0;
+    const __nv_bfloat16* take(size_t n) {
+        const __nv_bfloat16* p = base ? base + off : nullptr;
+        off = al128(off + n);
+        return p;
+    }
+};
+
+static void walk_attn(BlobWalk& w, size_t di, size_t d, const __nv_bfloat16*& q, const __nv_bfloat16*& k,
+                      const __nv_bfloat16*& v, const __nv_bfloat16*& o) {
+    q = w.take(di * d); k = w.take(di * d); v = w.take(di * d); o = w.take(d * di);
+}
+
+static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, csd_model* m) {
+    BlobWalk w{base};
+    const size_t d = c.d_model, di = (size_t)c.n_heads * c.d_head, ff = c.d_ff, V = c.vocab;
+    const __nv_bfloat16* embed = w.take(V * d);
+    std::vector<LayerW> enc, dec;
+    const __nv_bfloat16 *enc_bias = nullptr, *dec_bias = nullptr, *enc_final = nullptr;
+    if (c.arch == 1) {
+        enc_bias = w.take((size_t)c.rel_buckets * c.n_heads);
+        for (int l = 0; l < c.n_enc_layers; ++l) {
+            LayerW y{};
+            y.norm1 = w.take(d);
+            walk_attn(w, di, d, y.wq, y.wk, y.wv, y.wo);
+            y.norm2 = w.take(d); y.wgate = w.take(ff * d); y.wup = w.take(ff * d); y.wdown = w.take(d * ff);
+            enc.push_back(y);
+        }
+        enc_final = w.take(d);
+        dec_bias = w.take((size_t)c.rel_buckets * c.n_heads);
+    }
+    for (int l = 0; l < c.n_layers; ++l) {
+        LayerW y{};
+        y.norm1 = w.take(d);
+        walk_attn(w, di, d, y.wq, y.wk, y.wv, y.wo);
+        if (c.arch == 1) {
+            y.norm_x = w.take(d);
+            walk_attn(w, di, d, y.xq, y.xk, y.xv, y.xo);
+        }
+        y.norm2 = w.take(d); y.wgate = w.take(ff * d); y.wup = w.take(ff * d); y.wdown = w.take(d * ff);
+        dec.push_back(y);
+    }
+    const __nv_bfloat16* final_norm = w.take(d);
+    const __nv_bfloat16* lm_head = w.take(V * d);
+    if (m) {
+        m->embed = embed; m->enc = enc; m->dec = dec; m->enc_rel_bias = enc_bias; m->dec_rel_bias = dec_bias;
+        m->enc_final_norm = enc_final; m->final_norm = final_norm; m->lm_head = lm_head;
+    }
+    return w.off;
+}
+
+struct WsLayout {
+    size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
+        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, total;
+    size_t layer_kv, layer_x;
+};
+
+static WsLayout ws_layout(const csd_model_config& c) {
+    WsLayout L{};
+    const size_t d = c.d_model, H = c.n_heads, Dh = c.d_head, di = H * Dh, ff = c.d_ff, V = c.vocab;
+    const size_t R = CSD_MAX_ROWS;
+    size_t off = 0;
+    auto put = [&](size_t bytes) { size_t o = off; off = align_up(off + bytes, 256); return o; };
+    L.layer_kv = H * (size_t)c.max_seq * Dh;
+    L.kcache = put(c.n_layers * L.layer_kv * 2);
+    L.vcache = put(c.n_layers * L.layer_kv * 2);
+    L.x = put(R * d * 4);
+    L.qkv = put(R * 3 * di * 4);
+    L.attn = put(R * di * 4);
+    L.act = put(R * ff * 4);
+    size_t gp = 0, nmax = 0;
+    auto mat = [&](size_t N, size_t K, bool dual) {
+        size_t b = linear_scratch_bytes((int)R, (int)N, (int)K, dual);
+        if (b > gp) gp = b;
+        if (N > nmax) nmax = N;
+    };
+    mat(3 * di, d, false); mat(di, d, false); mat(d, di, false); mat(ff, d, true); mat(d, ff, false); mat(V, d, false);
+    L.gemm_partial = put(gp);
+    L.gemm_tickets = put((size_t)linear_ticket_count((int)nmax) * 4);
+    size_t keys = c.max_seq > c.max_enc_len ? c.max_seq : c.max_enc_len;
+    L.attn_partial = put(attn_scratch_bytes((int)keys, (int)H, (int)Dh));
+    L.attn_tickets = put(H * 4);
+    if (c.arch == 0) {
+        L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
+        L.rope_s = put((size_t)c.max_seq * (Dh / 2) * 4);
+    } else {
+        const size_t E = c.max_enc_len;
+        L.layer_x = H * E * Dh;
+        L.xk = put(c.n_layers * L.layer_x * 2);
+        L.xv = put(c.n_layers * L.layer_x * 2);
+        L.ek = put(L.layer_x * 2);
+        L.ev = put(L.layer_x * 2);
+        L.xenc = put(E * d * 4);
+        L.qkv_enc = put(E * 3 * di * 4);
+        L.dec_bias = put(H * (size_t)c.max_seq * 4);
+        L.enc_bias = put(H * (2 * E - 1) * 4);
+        L.buckets = put((c.max_seq + 2 * E) * 4);
+    }
+    L.total = off;
+    return L;
+}
+
+static csd_status check_config(const csd_model_config* c) {
+    if (!c) return CSD_ERR_INVALID_ARG;
+    if (c->arch != 0 && c->arch != 1) return CSD_ERR_UNSUPPORTED;
+    if (c->n_layers < 1 || c->d_model < 8 || c->n_heads < 1 || c->d_ff < 8 || c->vocab < 1 || c->max_seq < 1)
+        return CSD_ERR_INVALID_ARG;
+    if (c->max_rows < 1 || c->max_rows > CSD_MAX_ROWS) return CSD_ERR_INVALID_ARG;
+    if ((c->d_model & 7) || (c->d_ff & 7)) return CSD_ERR_SHAPE;
+    if (c->d_head != 32 && c->d_head != 64 && c->d_head != 128) return CSD_ERR_SHAPE;
+    if (c->arch == 1) {
+        if (c->n_enc_layers < 1 || c->max_enc_len < 1 || c->rel_buckets < 4 || (c->rel_buckets & 3) ||
+            c->rel_max_dist < c->rel_buckets)
+            return CSD_ERR_INVALID_ARG;
+    }
+    return CSD_OK;
+}
+
+// One linear layer of the forward; all of them share the model's split scratch.
+static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat16* W2, int N, int K, const float* X,
+                         int ldx, int m, const __nv_bfloat16* gain, float* Y, int ldy, int epi, cudaStream_t st) {
+    LinearArgs a;
+    a.W = W; a.W2 = W2; a.N = N; a.K = K; a.X = X; a.ldx = ldx; a.m = m; a.gain = gain; a.eps = M->cfg.norm_eps;
+    a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.partial = M->gemm_partial; a.tickets = M->gemm_tickets;
+    return launch_linear(a, st);
+}
+
+#define CSD_TRY(expr)                       \
+    do {                                    \
+        csd_status s__ = (expr);            \
+        if (s__ != CSD_OK) return s__;      \
+    } while (0)
+
+// q|k|v projections of `m` rows with the norm fused; one GEMM when the three matrices are
+// contiguous in the blob (they are whenever d_inner * d_model is a multiple of 128).
+static csd_status project_qkv(csd_model* M, const LayerW& y, const float* X, int m, float* out, cudaStream_t st) {
+    const int d = M->cfg.d_model, di = M->di;
+    if (y.wk == y.wq + (size_t)di * d && y.wv == y.wk + (size_t)di * d)
+        return linear(M, y.wq, nullptr, 3 * di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st);
+    CSD_TRY(linear(M, y.wq, nullptr, di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st));
+    CSD_TRY(linear(M, y.wk, nullptr, di, d, X, d, m, y.norm1, out + di, 3 * di, EPI_STORE, st));
+    return linear(M, y.wv, nullptr, di, d, X, d, m, y.norm1, out + 2 * di, 3 * di, EPI_STORE, st);
+}
+
+static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, cudaStream_t st) {
+    const int d = M->cfg.d_model, ff = M->cfg.d_ff;
+    CSD_TRY(linear(M, y.wgate, y.wup, ff, d, X, d, m, y.norm2, M->act, ff, M->cfg.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, st));
+    return linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, X, d, EPI_ADD, st);
+}
+
+}  // namespace csd
+
+using namespace csd;
+
+extern "C" int csd_rel_bucket(int rel, int bidirectional, int n_buckets, int max_dist) {
+    int bucket = 0, B = n_buckets, n;
+    if (bidirectional) {
+        B /= 2;
+        if (rel > 0) bucket += B;
+        n = rel < 0 ? -rel : rel;
+    } else {
+        n = rel < 0 ? -rel : 0;
+    }
+    const int exact = B / 2;
+    if (n < exact) return bucket + n;
+    // logarithmic part; the tiny nudge keeps distances that sit exactly on a bucket edge
+    // (powers of two) on the upper side, as exact arithmetic puts them
+    double t = log((double)n / exact) / log((double)max_dist / exact) * (B - exact);
+    int b = exact + (int)floor(t + 1e-9);
+    if (b > B - 1) b = B - 1;
+    return bucket + b;
+}
+
+extern "C" size_t csd_model_weight_bytes(const csd_model_config* cfg) {
+    if (check_config(cfg) != CSD_OK) return 0;
+    return walk_blob(*cfg, nullptr, nullptr) * sizeof(__nv_bfloat16);
+}
+
+extern "C" size_t csd_model_workspace_bytes(const csd_model_config* cfg) {
+    if (check_config(cfg) != CSD_OK) return 0;
+    return ws_layout(*cfg).total;
+}
+
+extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* weights_bf16_dev, size_t weight_bytes,
+                                       void* workspace_dev, size_t workspace_bytes, void* stream, csd_model** out) {
+    if (!out) return CSD_ERR_INVALID_ARG;
+    *out = nullptr;
+    CSD_TRY(check_config(cfg));
+    if (!weights_bf16_dev || !workspace_dev) return CSD_ERR_INVALID_ARG;
+    if ((((uintptr_t)weights_bf16_dev) & 255) || (((uintptr_t)workspace_dev) & 255)) return CSD_ERR_INVALID_ARG;
+    if (weight_bytes < csd_model_weight_bytes(cfg)) return CSD_ERR_CAPACITY;
+    const WsLayout L = ws_layout(*cfg);
+    if (workspace_bytes < L.total) return CSD_ERR_CAPACITY;
+    int* status = status_word_device();
+    if (!status) return CSD_ERR_CUDA;
+    csd_model* M = new (std::nothrow) csd_model();
+    if (!M) return CSD_ERR_OOM;
+    M->cfg = *cfg;
+    M->di = cfg->n_heads * cfg->d_head;
+    walk_blob(*cfg, (const __nv_bfloat16*)weights_bf16_dev, M);
+    char* ws = (char*)workspace_dev;
+    M->kcache = (__nv_bfloat16*)(ws + L.kcache); M->vcache = (__nv_bfloat16*)(ws + L.vcache);
+    M->layer_kv = L.layer_kv; M->layer_x = L.layer_x;
+    M->x = (float*)(ws + L.x); M->qkv = (float*)(ws + L.qkv); M->attn = (float*)(ws + L.attn);
+    M->act = (float*)(ws + L.act);
+    M->gemm_partial = (float*)(ws + L.gemm_partial); M->gemm_tickets = (unsigned*)(ws + L.gemm_tickets);
+    M->attn_partial = (float*)(ws + L.attn_partial); M->attn_tickets = (unsigned*)(ws + L.attn_tickets);
+    M->status = status;
+    cudaStream_t st = (cudaStream_t)stream;
+    cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.attn_partial - L.gemm_tickets, st);
+    if (e == cudaSuccess) e = cudaMemsetAsync(ws + L.attn_tickets, 0, (size_t)cfg->n_heads * 4, st);
+    if (e != cudaSuccess) { delete M; return note_cuda(e); }
+    if (cfg->arch == 0) {
+        M->rope_c = (float*)(ws + L.rope_c); M->rope_s = (float*)(ws + L.rope_s);
+        const int n = cfg->max_seq * (cfg->d_head / 2);
+        rope_table_kernel<<<(n + 255) / 256, 256, 0, st>>>(M->rope_c, M->rope_s, cfg->max_seq, cfg->d_head / 2,
+                                                           (double)cfg->rope_theta);
+        count_launch();
+    } else {
+        const int E = cfg->max_enc_len, S = cfg->max_seq;
+        M->xk = (__nv_bfloat16*)(ws + L.xk); M->xv = (__nv_bfloat16*)(ws + L.xv);
+        M->ek = (__nv_bfloat16*)(ws + L.ek); M->ev = (__nv_bfloat16*)(ws + L.ev);
+        M->xenc = (float*)(ws + L.xenc); M->qkv_enc = (float*)(ws + L.qkv_enc);
+        M->dec_bias = (float*)(ws + L.dec_bias); M->enc_bias = (float*)(ws + L.enc_bias);
+        int* buckets = (int*)(ws + L.buckets);
+        std::vector<int> hb((size_t)S + 2 * E - 1);
+        // decoder: index i <-> rel = i - (S-1) in [-(S-1), 0]; encoder: rel = i - (E-1) in [-(E-1), E-1]
+        for (int i = 0; i < S; ++i) hb[i] = csd_rel_bucket(i - (S - 1), 0, cfg->rel_buckets, cfg->rel_max_dist);
+        for (int i = 0; i < 2 * E - 1; ++i)
+            hb[S + i] = csd_rel_bucket(i - (E - 1), 1, cfg->rel_buckets, cfg->rel_max_dist);
+        e = cudaMemcpyAsync(buckets, hb.data(), hb.size() * sizeof(int), cudaMemcpyHostToDevice, st);
+        if (e == cudaSuccess) e = cudaStreamSynchronize(st);   // hb goes out of scope below
+        if (e != cudaSuccess) { delete M; return note_cuda(e); }
+        bias_table_kernel<<<(S * cfg->n_heads + 255) / 256, 256, 0, st>>>(M->dec_rel_bias, buckets, S, cfg->n_heads, M->dec_bias);
+        bias_table_kernel<<<((2 * E - 1) * cfg->n_heads + 255) / 256, 256, 0, st>>>(M->enc_rel_bias, buckets + S, 2 * E - 1,
+                                                                                 cfg->n_heads, M->enc_bias);
+        count_launch(2);
+    }
+    e = cudaGetLastError();
+    if (e != cudaSuccess) { delete M; return note_cuda(e); }
+    *out = M;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_model_destroy(csd_model* m) {
+    delete m;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_tokens_dev, int n, void* stream) {
+    if (!M || !enc_tokens_dev) return CSD_ERR_INVALID_ARG;
+    const csd_model_config& c = M->cfg;
+    if (c.arch != 1) return CSD_ERR_UNSUPPORTED;
+    if (n < 1 || n > c.max_enc_len) return CSD_ERR_CAPACITY;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, E = c.max_enc_len;
+    const int CH = 16;
+    embed_kernel<<<n, 128, 0, st>>>(enc_tokens_dev, M->embed, c.vocab, d, M->xenc, M->status);
+    count_launch();
+    for (int l = 0; l < c.n_enc_layers; ++l) {
+        const LayerW& y = M->enc[l];
+        for (int r0 = 0; r0 < n; r0 += CH) {
+            const int m = n - r0 < CH ? n - r0 : CH;
+            CSD_TRY(project_qkv(M, y, M->xenc + (size_t)r0 * d, m, M->qkv_enc + (size_t)r0 * 3 * di, st));
+        }
+        rope_append_kernel<<<dim3(n, H), 64, 0, st>>>(M->qkv_enc, 3 * di, -1, di, 2 * di, Dh, 0, E, nullptr, nullptr,
+                                                      M->ek, M->ev);
+        count_launch();
+        for (int r0 = 0; r0 < n; r0 += CH) {
+            const int m = n - r0 < CH ? n - r0 : CH;
+            AttnArgs a;
+            a.q = M->qkv_enc + (size_t)r0 * 3 * di; a.ldq = 3 * di; a.m = m; a.Kc = M->ek; a.Vc = M->ev; a.cap = E;
+            a.H = H; a.Dh = Dh; a.n_keys = n; a.causal = 0; a.scale = 1.f; a.bias = M->enc_bias;
+            a.bias_len = 2 * E - 1; a.bias_zero = E - 1; a.q_pos0 = r0; a.out = M->attn; a.ldo = di;
+            a.partial = M->attn_partial; a.tickets = M->attn_tickets;
+            CSD_TRY(launch_attention(a, st));
+            float* xr = M->xenc + (size_t)r0 * d;
+            CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, xr, d, EPI_ADD, st));
+            CSD_TRY(feed_forward(M, y, xr, m, st));
+        }
+    }
+    // static cross-attention K/V of every decoder layer from the normed encoder output
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerW& y = M->dec[l];
+        for (int r0 = 0; r0 < n; r0 += CH) {
+            const int m = n - r0 < CH ? n - r0 : CH;
+            const float* xr = M->xenc + (size_t)r0 * d;
+            float* o = M->qkv_enc + (size_t)r0 * 3 * di;
+            CSD_TRY(linear(M, y.xk, nullptr, di, d, xr, d, m, M->enc_final_norm, o + di, 3 * di, EPI_STORE, st));
+            CSD_TRY(linear(M, y.xv, nullptr, di, d, xr, d, m, M->enc_final_norm, o + 2 * di, 3 * di, EPI_STORE, st));
+        }
+        rope_append_kernel<<<dim3(n, H), 64, 0, st>>>(M->qkv_enc, 3 * di, -1, di, 2 * di, Dh, 0, E, nullptr, nullptr,
+                                                      M->xk + (size_t)l * M->layer_x, M->xv + (size_t)l * M->layer_x);
+        count_launch();
+    }
+    CSD_CUDA(cudaGetLastError());
+    M->enc_len = n;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
+                                         float* logits_out_dev, void* stream) {
+    if (!M || !block_tokens_dev || !logits_out_dev) return CSD_ERR_INVALID_ARG;
+    const csd_model_config& c = M->cfg;
+    if (m < 1 || m > c.max_rows || kv_len < 0) return CSD_ERR_INVALID_ARG;
+    if (kv_len + m > c.max_seq) return CSD_ERR_CAPACITY;
+    if (c.arch == 1 && M->enc_len < 1) return CSD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, V = c.vocab;
+    embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
+    count_launch();
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerW& y = M->dec[l];
+        __nv_bfloat16* Kl = M->kcache + (size_t)l * M->layer_kv;
+        __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
+        CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st));
+        rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
+                                                      c.arch == 0 ? M->rope_c : nullptr, c.arch == 0 ? M->rope_s : nullptr,
+                                                      Kl, Vl);
+        count_launch();
+        AttnArgs a;
+        a.q = M->qkv; a.ldq = 3 * di; a.m = m; a.Kc = Kl; a.Vc = Vl; a.cap = c.max_seq; a.H = H; a.Dh = Dh;
+        a.n_keys = kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
+        if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = kv_len; }
+        a.out = M->attn; a.ldo = di; a.partial = M->attn_partial; a.tickets = M->attn_tickets;
+        CSD_TRY(launch_attention(a, st));
+        CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
+        if (c.arch == 1) {
+            CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st));
+            AttnArgs x;
+            x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
+            x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
+            x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di; x.partial = M->attn_partial;
+            x.tickets = M->attn_tickets;
+            CSD_TRY(launch_attention(x, st));
+            CSD_TRY(linear(M, y.xo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
+        }
+        CSD_TRY(feed_forward(M, y, M->x, m, st));
+    }
+    CSD_TRY(linear(M, M->lm_head, nullptr, V, d, M->x, d, m, M->final_norm, logits_out_dev, V, EPI_STORE, st));
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
+}

@@ -1,0 +1,31 @@
+// Model handle shared by model.cu and cascade.cu.
+#pragma once
+#include <vector>
+#include "attention.cuh"
+#include "common.cuh"
+#include "gemm.cuh"
+
+namespace csd {
+struct LayerW {
+    const __nv_bfloat16 *norm1, *wq, *wk, *wv, *wo, *norm_x, *xq, *xk, *xv, *xo, *norm2, *wgate, *wup, *wdown;
+};
+}  // namespace csd
+
+struct csd_model {
+    csd_model_config cfg;
+    int di = 0;                 // n_heads * d_head
+    int enc_len = 0;            // encoder positions cached by csd_encoder_forward
+    const __nv_bfloat16 *embed = nullptr, *final_norm = nullptr, *lm_head = nullptr, *enc_rel_bias = nullptr,
+                        *dec_rel_bias = nullptr, *enc_final_norm = nullptr;
+    std::vector<csd::LayerW> enc, dec;
+    // workspace views
+    __nv_bfloat16 *kcache = nullptr, *vcache = nullptr;   // [layer][head][max_seq][Dh]
+    __nv_bfloat16 *xk = nullptr, *xv = nullptr;           // cross K/V [layer][head][max_enc_len][Dh]
+    __nv_bfloat16 *ek = nullptr, *ev = nullptr;           // encoder self K/V of the layer in flight
+    size_t layer_kv = 0, layer_x = 0;
+    float *x = nullptr, *qkv = nullptr, *attn = nullptr, *act = nullptr, *xenc = nullptr, *qkv_enc = nullptr;
+    float *rope_c = nullptr, *rope_s = nullptr, *dec_bias = nullptr, *enc_bias = nullptr;
+    float *gemm_partial = nullptr, *attn_partial = nullptr;
+    unsigned *gemm_tickets = nullptr, *attn_tickets = nullptr;
+    int* status = nullptr;
+};
