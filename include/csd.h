@@ -118,6 +118,23 @@ csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int 
 csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
                               float* logits_out_dev, void* stream);
 
+/* Per-kernel-class timing of later forwards of this model (measurement aid; the paper's unit of
+ * cost is "a single run" of a model, Section 4).  While enabled, every kernel launch of
+ * csd_review_forward is bracketed by a CUDA event pair on the launching stream (a few
+ * microseconds of overhead per launch).  csd_model_profile_read waits for the stream, sums the
+ * pairs recorded since the last read per class and clears them. */
+typedef struct {
+    double gemm_ms;            /* weight-streaming GEMM launches                    */
+    int64_t gemm_launches;
+    double gemm_weight_bytes;  /* bf16 weight bytes those launches streamed         */
+    double attn_ms;            /* block-attention launches                          */
+    int64_t attn_launches;
+    double other_ms;           /* embedding gather, rotary + K/V append             */
+    int64_t other_launches;
+} csd_profile;
+csd_status csd_model_profile(csd_model* m, int enable);
+csd_status csd_model_profile_read(csd_model* m, void* stream, csd_profile* out);
+
 /* Y[m, N] = X[m, K] . W[N, K]^T, the weight-streaming contraction every layer of the review
  * forward is made of (W bf16 row-major, X and Y fp32 row-major, fp32 accumulation).  Exposed
  * for kernel-level tests and roofline measurements.  1 <= m <= 17, K multiple of 8. */

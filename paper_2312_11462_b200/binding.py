@@ -57,6 +57,12 @@ class CascadeStats(C.Structure):
                     total_ms=self.total_ms)
 
 
+class Profile(C.Structure):
+    _fields_ = [("gemm_ms", C.c_double), ("gemm_launches", C.c_int64), ("gemm_weight_bytes", C.c_double),
+                ("attn_ms", C.c_double), ("attn_launches", C.c_int64), ("other_ms", C.c_double),
+                ("other_launches", C.c_int64)]
+
+
 _vp, _i, _sz, _f, _u64 = C.c_void_p, C.c_int, C.c_size_t, C.c_float, C.c_uint64
 lib.csd_status_string.restype = C.c_char_p
 lib.csd_status_string.argtypes = [_i]
@@ -70,6 +76,8 @@ lib.csd_model_create.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _vp]
 lib.csd_model_destroy.argtypes = [_vp]
 lib.csd_encoder_forward.argtypes = [_vp, _vp, _i, _vp]
 lib.csd_review_forward.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
+lib.csd_model_profile.argtypes = [_vp, _i]
+lib.csd_model_profile_read.argtypes = [_vp, _vp, _vp]
 lib.csd_linear_workspace_bytes.restype = _sz
 lib.csd_linear_workspace_bytes.argtypes = [_i, _i, _i]
 lib.csd_linear.argtypes = [_vp, _i, _i, _vp, _i, _vp, _vp, _sz, _vp]
@@ -153,6 +161,14 @@ class Model:
         _check("csd_review_forward",
                lib.csd_review_forward(self.h, _ptr(block_tokens), m, kv_len, _ptr(logits_out), _stream()))
         return logits_out
+
+    def csd_model_profile(self, enable: bool) -> None:
+        _check("csd_model_profile", lib.csd_model_profile(self.h, int(enable)))
+
+    def csd_model_profile_read(self) -> dict:
+        p = Profile()
+        _check("csd_model_profile_read", lib.csd_model_profile_read(self.h, _stream(), C.byref(p)))
+        return {n: getattr(p, n) for n, _ in Profile._fields_}
 
     def close(self) -> None:
         if getattr(self, "h", None):

@@ -4,6 +4,7 @@
 #include <math.h>
 #include <new>
 #include <stdlib.h>
+#include <string.h>
 #include <vector>
 
 namespace csd {
@@ -202,6 +203,8 @@ static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat
     LinearArgs a;
     a.W = W; a.W2 = W2; a.N = N; a.K = K; a.X = X; a.ldx = ldx; a.m = m; a.gain = gain; a.eps = M->cfg.norm_eps;
     a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.partial = M->gemm_partial; a.tickets = M->gemm_tickets;
+    ProfScope ps(M, 0, st);
+    if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
     return launch_linear(a, st);
 }
 
@@ -210,6 +213,11 @@ static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat
         csd_status s__ = (expr);            \
         if (s__ != CSD_OK) return s__;      \
     } while (0)
+
+static csd_status attention(csd_model* M, const AttnArgs& a, cudaStream_t st) {
+    ProfScope ps(M, 1, st);
+    return launch_attention(a, st);
+}
 
 // q|k|v projections of `m` rows with the norm fused; one GEMM when the three matrices are
 // contiguous in the blob (they are whenever d_inner * d_model is a multiple of 128).
@@ -323,7 +331,37 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
 }
 
 extern "C" csd_status csd_model_destroy(csd_model* m) {
+    if (m)
+        for (cudaEvent_t e : m->prof_ev) cudaEventDestroy(e);
     delete m;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_model_profile(csd_model* m, int enable) {
+    if (!m) return CSD_ERR_INVALID_ARG;
+    m->prof = enable != 0;
+    m->prof_used = 0;
+    m->prof_gemm_bytes = 0.0;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_model_profile_read(csd_model* m, void* stream, csd_profile* out) {
+    if (!m || !out) return CSD_ERR_INVALID_ARG;
+    CSD_CUDA(cudaStreamSynchronize((cudaStream_t)stream));
+    csd_profile p;
+    memset(&p, 0, sizeof(p));
+    for (size_t i = 0; i < m->prof_used; ++i) {
+        float ms = 0.f;
+        CSD_CUDA(cudaEventElapsedTime(&ms, m->prof_ev[2 * i], m->prof_ev[2 * i + 1]));
+        const int k = m->prof_kind[i];
+        if (k == 0) { p.gemm_ms += ms; p.gemm_launches += 1; }
+        else if (k == 1) { p.attn_ms += ms; p.attn_launches += 1; }
+        else { p.other_ms += ms; p.other_launches += 1; }
+    }
+    p.gemm_weight_bytes = m->prof_gemm_bytes;
+    m->prof_used = 0;
+    m->prof_gemm_bytes = 0.0;
+    *out = p;
     return CSD_OK;
 }
 
@@ -353,7 +391,7 @@ extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_token
             a.H = H; a.Dh = Dh; a.n_keys = n; a.causal = 0; a.scale = 1.f; a.bias = M->enc_bias;
             a.bias_len = 2 * E - 1; a.bias_zero = E - 1; a.q_pos0 = r0; a.out = M->attn; a.ldo = di;
             a.partial = M->attn_partial; a.tickets = M->attn_tickets;
-            CSD_TRY(launch_attention(a, st));
+            CSD_TRY(attention(M, a, st));
             float* xr = M->xenc + (size_t)r0 * d;
             CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, xr, d, EPI_ADD, st));
             CSD_TRY(feed_forward(M, y, xr, m, st));
@@ -387,23 +425,29 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
     if (c.arch == 1 && M->enc_len < 1) return CSD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, V = c.vocab;
-    embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
-    count_launch();
+    {
+        ProfScope ps(M, 2, st);
+        embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
+        count_launch();
+    }
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& y = M->dec[l];
         __nv_bfloat16* Kl = M->kcache + (size_t)l * M->layer_kv;
         __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
         CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st));
-        rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
-                                                      c.arch == 0 ? M->rope_c : nullptr, c.arch == 0 ? M->rope_s : nullptr,
-                                                      Kl, Vl);
-        count_launch();
+        {
+            ProfScope ps(M, 2, st);
+            rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
+                                                          c.arch == 0 ? M->rope_c : nullptr,
+                                                          c.arch == 0 ? M->rope_s : nullptr, Kl, Vl);
+            count_launch();
+        }
         AttnArgs a;
         a.q = M->qkv; a.ldq = 3 * di; a.m = m; a.Kc = Kl; a.Vc = Vl; a.cap = c.max_seq; a.H = H; a.Dh = Dh;
         a.n_keys = kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
         if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = kv_len; }
         a.out = M->attn; a.ldo = di; a.partial = M->attn_partial; a.tickets = M->attn_tickets;
-        CSD_TRY(launch_attention(a, st));
+        CSD_TRY(attention(M, a, st));
         CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
         if (c.arch == 1) {
             CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st));
@@ -412,7 +456,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
             x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
             x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di; x.partial = M->attn_partial;
             x.tickets = M->attn_tickets;
-            CSD_TRY(launch_attention(x, st));
+            CSD_TRY(attention(M, x, st));
             CSD_TRY(linear(M, y.xo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
         }
         CSD_TRY(feed_forward(M, y, M->x, m, st));

@@ -28,4 +28,32 @@ struct csd_model {
     float *gemm_partial = nullptr, *attn_partial = nullptr;
     unsigned *gemm_tickets = nullptr, *attn_tickets = nullptr;
     int* status = nullptr;
+    // optional per-kernel-class timing (csd_model_profile): event pairs around every launch
+    bool prof = false;
+    std::vector<cudaEvent_t> prof_ev;      // start, stop, start, stop, ...
+    std::vector<int> prof_kind;            // class of each pair: 0 GEMM, 1 attention, 2 other
+    size_t prof_used = 0;                  // pairs recorded since the last read
+    double prof_gemm_bytes = 0.0;          // weight bytes the recorded GEMM launches streamed
 };
+
+namespace csd {
+// Records an event pair around the launches made during its lifetime when profiling is on.
+struct ProfScope {
+    csd_model* M; cudaStream_t st; bool on;
+    ProfScope(csd_model* m, int kind, cudaStream_t s) : M(m), st(s), on(m->prof) {
+        if (!on) return;
+        if (M->prof_used * 2 + 2 > M->prof_ev.size()) {
+            cudaEvent_t a = nullptr, b = nullptr;
+            if (cudaEventCreate(&a) != cudaSuccess || cudaEventCreate(&b) != cudaSuccess) { on = false; return; }
+            M->prof_ev.push_back(a); M->prof_ev.push_back(b); M->prof_kind.push_back(kind);
+        }
+        M->prof_kind[M->prof_used] = kind;
+        cudaEventRecord(M->prof_ev[M->prof_used * 2], st);
+    }
+    ~ProfScope() {
+        if (!on) return;
+        cudaEventRecord(M->prof_ev[M->prof_used * 2 + 1], st);
+        M->prof_used += 1;
+    }
+};
+}  // namespace csd

@@ -1,0 +1,115 @@
+"""Parity of csd_spec_accept with the oracle: accepted count and output token bit-exact on every
+row the oracle does not flag as a near tie (those are counted and must be rare)."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from gpu_util import require_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    require_gpu()
+    from paper_2312_11462_b200 import binding
+    return binding
+
+
+def compare(b, orc, t, d, tok, temperature, lenience=1.0, seed=7, step=3, onehot=None, max_flag_frac=0.02):
+    tn = t.cpu().numpy()
+    dn = None if d is None else d.cpu().numpy()
+    on = None if onehot is None else onehot.cpu().numpy()
+    n_ref, o_ref, flags = orc.spec_accept(tn, dn, tok.cpu().numpy(), temperature, lenience, seed, step, onehot=on)
+    n, o = b.csd_spec_accept(t, d, tok, temperature, lenience, seed, step, onehot=onehot)
+    assert b.csd_device_status() == 0
+    n, o = n.cpu().numpy(), o.cpu().numpy()
+    ok = flags == 0
+    assert (~ok).mean() <= max_flag_frac, f"{(~ok).sum()} of {len(ok)} rows flagged as near ties"
+    bad = np.nonzero(ok & ((n != n_ref) | (o != o_ref)))[0]
+    assert bad.size == 0, (bad[:5], n[bad[:5]], n_ref[bad[:5]], o[bad[:5]], o_ref[bad[:5]])
+    # flagged rows must still be valid outcomes
+    assert ((n >= 0) & (n <= t.shape[1] - 1)).all() and ((o >= 0) & (o < t.shape[2])).all()
+    return n_ref, o_ref
+
+
+@pytest.mark.parametrize("V", [4096, 32000, 128256])
+@pytest.mark.parametrize("k", [1, 4, 16])
+@pytest.mark.parametrize("sigma", [0.1, 0.5, 2.0])
+def test_sampling_sweep(b, orc, V, k, sigma):
+    rows = 64 if V < 100000 else 16      # the oracle's cost is what bounds the big-vocabulary case
+    t, d, tok = workloads.accept_case(rows, k, V, sigma, seed=V + 31 * k, device="cuda")
+    n_ref, _ = compare(b, orc, t, d, tok, 1.0)
+    if sigma == 0.1:
+        assert n_ref.mean() > 0.5 * k       # close drafts are mostly accepted
+
+
+@pytest.mark.parametrize("V,k", [(4096, 2), (32000, 8), (128256, 16)])
+def test_greedy(b, orc, V, k):
+    t, d, tok = workloads.accept_case(64, k, V, 0.1, seed=5, device="cuda")
+    am = t.argmax(-1)[:, :k].to(torch.int32)
+    cut = torch.arange(64, device="cuda") % (k + 1)
+    tok = am.clone()
+    for r in range(64):
+        if cut[r] < k:
+            tok[r, cut[r]] = (tok[r, cut[r]] + 1) % V
+    n, o = compare(b, orc, t, None, tok.contiguous(), 0.0)
+    assert (n == cut.cpu().numpy()).all()
+
+
+def test_ragged_vocab_and_edge_cases(b, orc):
+    # vocabulary sizes that are not multiples of the vector width or of a chunk
+    for V in (8, 1000, 4097, 50257):
+        for k in (0, 1, 3):
+            t, d, tok = workloads.accept_case(33, k, V, 1.0, seed=V + k, device="cuda")
+            compare(b, orc, t, d, tok, 1.0)
+            compare(b, orc, t, None, tok, 1.0)          # point-mass drafts
+            compare(b, orc, t, d, tok, 0.0)             # greedy
+    # temperature and lenience
+    t, d, tok = workloads.accept_case(64, 4, 5000, 1.0, seed=2, device="cuda")
+    compare(b, orc, t, d, tok, 0.7)
+    compare(b, orc, t, d, tok, 1.3, lenience=3.0)
+    # mixed block: some positions come from a statistical drafter
+    onehot = (torch.arange(64 * 4, device="cuda").reshape(64, 4) % 3 == 0).to(torch.int32)
+    compare(b, orc, t, d, tok, 1.0, onehot=onehot)
+    # q == p: everything accepted, bonus token from the last law
+    n, _ = compare(b, orc, t, t[:, :4].contiguous(), tok, 1.0)
+    assert (n == 4).all()
+    # -inf logits (masked vocabulary entries)
+    t2 = t.clone()
+    t2[:, :, ::2] = float("-inf")
+    compare(b, orc, t2, d, tok, 1.0)
+    # unaligned base pointers take the scalar path
+    buf = torch.zeros(64 * 5 * 5000 + 1, device="cuda")
+    tu = buf[1:].view(64, 5, 5000)
+    tu.copy_(t)
+    compare(b, orc, tu, d, tok, 1.0)
+
+
+def test_bad_token_sets_status(b):
+    t, d, tok = workloads.accept_case(4, 2, 512, 1.0, seed=1, device="cuda")
+    tok[2, 0] = 512
+    n, o = b.csd_spec_accept(t, d, tok, 1.0)
+    assert b.csd_device_status() == 6
+    assert b.csd_device_status() == 0          # reading clears it
+    assert int(n[2]) == 0
+
+
+def test_distribution_on_tiny_vocab(b, orc):
+    # the kernel's own draws reproduce the target law (chi-square, p > 0.01)
+    from scipy import stats
+    V, k, N = 8, 2, 200_000
+    tl, dl = workloads.small_logits(1, k, V, seed=11, scale=1.5)
+    p = np.exp(tl[0].astype(np.float64)); p /= p.sum(-1, keepdims=True)
+    q = np.exp(dl[0].astype(np.float64)); q /= q.sum(-1, keepdims=True)
+    rng = np.random.default_rng(0)
+    tok = np.stack([rng.choice(V, size=N, p=q[i]) for i in range(k)], axis=1).astype(np.int32)
+    t = torch.from_numpy(np.broadcast_to(tl[0], (N, k + 1, V)).copy()).cuda()
+    d = torch.from_numpy(np.broadcast_to(dl[0], (N, k, V)).copy()).cuda()
+    n, o = b.csd_spec_accept(t, d, torch.from_numpy(tok).cuda(), 1.0, seed=99)
+    n, o = n.cpu().numpy(), o.cpu().numpy()
+    y1 = np.where(n >= 1, tok[:, 0], o)
+    assert stats.chisquare(np.bincount(y1, minlength=V), p[0] * N).pvalue > 0.01
+    y3 = o[n == 2]
+    assert stats.chisquare(np.bincount(y3, minlength=V), p[2] * len(y3)).pvalue > 0.01

@@ -1,0 +1,68 @@
+"""Parity at the workloads' own sizes: the 7B-shaped target with its 68M-shaped draft (cascade
+on a short prompt, because the oracle needs ~6 s of host time per target row block), and the
+long-cache review (2048+ cached positions, head dimension 128, blocks of 2/5/9/17 rows) on a
+narrower model that the oracle can prefill in seconds."""
+import numpy as np
+import pytest
+import torch
+
+import workloads
+from workloads import SHAPES, llama_shape
+from gpu_util import LOGIT_MAX_ABS, LOGIT_REL_L2, rel_l2, require_gpu, to_dev_i32
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    require_gpu()
+    from paper_2312_11462_b200 import binding
+    return binding
+
+
+def test_7b_shaped_cascade_and_logits(b, orc):
+    ts, ds = SHAPES["llama7b"], SHAPES["draft68m"]
+    tb = workloads.make_weights(ts, seed=100, device="cuda")
+    db = workloads.make_weights(ds, seed=101, device="cuda")
+    prompt = workloads.make_prompt(ts.vocab, 12, seed=1000)
+    nxt = workloads.bigram_table(prompt, ts.vocab, seed=7)
+    K, max_block, n_new = [[4, 0], [0, 4]], 4, 6
+    oms = [orc.Model(ts, orc.blob_to_u16(tb)), orc.Model(ds, orc.blob_to_u16(db))]
+    want, margins, ost = orc.cascade_generate(oms, prompt, nxt, K, max_block, prompt, n_new)
+    gms = [b.Model(ts, tb), b.Model(ds, db)]
+    got, st = b.Cascade(gms, K, max_block, to_dev_i32(nxt), 128).csd_cascade_generate(prompt, prompt, n_new)
+    low = np.nonzero(margins < 0.05)[0]
+    safe = int(low[0]) if low.size else n_new
+    assert list(got[:safe]) == list(want[:safe])
+    assert b.csd_device_status() == 0
+    # teacher-forced: the target's logits over the oracle's own sequence, block by block
+    seq = np.concatenate([prompt, want]).astype(np.int32)
+    gm, om = gms[0], orc.Model(ts, orc.blob_to_u16(tb))
+    for pos, m in ((0, 11), (11, 5), (16, 2)):
+        blk = seq[pos:pos + m]
+        g = gm.csd_review_forward(to_dev_i32(blk), pos).cpu().numpy()
+        r = om.review_forward(blk, pos)
+        assert rel_l2(g, r) <= LOGIT_REL_L2, (pos, rel_l2(g, r))
+        assert np.abs(g - r).max() <= LOGIT_MAX_ABS
+
+
+def test_long_cache_review_blocks(b, orc):
+    shape = llama_shape(2, 1024, 8, 2752, 8000, 2624)
+    blob = workloads.make_weights(shape, seed=21, device="cuda")
+    toks = workloads.make_prompt(shape.vocab, 2100, seed=3)
+    gm, om = b.Model(shape, blob), orc.Model(shape, orc.blob_to_u16(blob))
+    S = 2048
+    for pos in range(0, S, 512):
+        om.review_forward(toks[pos:pos + 512], pos)
+    pos = 0
+    while pos < S:
+        n = min(16, S - pos)
+        gm.csd_review_forward(to_dev_i32(toks[pos:pos + n]), pos)
+        pos += n
+    for m in (2, 5, 9, 17):
+        blk = toks[S:S + m]
+        g = gm.csd_review_forward(to_dev_i32(blk), S).cpu().numpy()
+        r = om.review_forward(blk, S)
+        assert rel_l2(g, r) <= LOGIT_REL_L2, (m, rel_l2(g, r))
+        assert np.abs(g - r).max() <= LOGIT_MAX_ABS
+    assert b.csd_device_status() == 0

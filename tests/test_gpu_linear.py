@@ -1,0 +1,44 @@
+"""Parity of the weight-streaming skinny GEMM (csd_linear) with the oracle's contraction."""
+import numpy as np
+import pytest
+import torch
+
+from gpu_util import rel_l2, require_gpu
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def b():
+    require_gpu()
+    from paper_2312_11462_b200 import binding
+    return binding
+
+
+def case(b, orc, m, N, K, seed):
+    g = torch.Generator(device="cuda")
+    g.manual_seed(seed)
+    W = (0.05 * torch.randn(N, K, generator=g, device="cuda")).to(torch.bfloat16)
+    X = torch.randn(m, K, generator=g, device="cuda")
+    Y = b.csd_linear(W, X)
+    Y2 = b.csd_linear(W, X)                      # split-K partials are summed in a fixed order
+    assert torch.equal(Y, Y2)
+    ref = orc.linear(orc.blob_to_u16(W).reshape(N, K), X.cpu().numpy())
+    got = Y.cpu().numpy()
+    # fp32 accumulation of K products of magnitude |w||x|: error ~ sqrt(K) * 2^-24 * |y|
+    assert rel_l2(got, ref) < 2e-6, (m, N, K)
+    assert np.abs(got - ref).max() < 1e-4 * max(1.0, np.abs(ref).max())
+
+
+@pytest.mark.parametrize("m", [1, 2, 5, 8, 9, 16, 17])
+def test_layer_shapes(b, orc, m):
+    # the matrix shapes of the small models plus ragged ones (N not a tile multiple, K one
+    # partial step, K with a tail slice)
+    for N, K in ((768, 768), (2304, 768), (4096, 256), (256, 1024), (64, 64), (1000, 136), (37, 2056), (4099, 520)):
+        case(b, orc, m, N, K, seed=N + K + m)
+
+
+@pytest.mark.parametrize("N,K", [(4096, 4096), (12288, 4096), (4096, 11008)])
+def test_7b_layer_shapes(b, orc, N, K):
+    for m in (5, 17):
+        case(b, orc, m, N, K, seed=m)
