@@ -2,12 +2,15 @@
 //
 // Every bf16 weight is read from HBM exactly once with 128-bit streaming loads and used for m
 // fused multiply-adds on the CUDA cores (fp32 accumulation), so for small m the kernel is bound
-// by HBM bandwidth.  Work is cut into units of (TN output columns) x (one K slice); a CTA takes
-// one unit, keeps its X slice in shared memory, and each warp streams R weight rows at a time.
-// With more than one K slice the CTAs leave fp32 partial tiles in scratch and the CTA that
-// arrives last at the tile's ticket adds them in slice order (deterministic) and runs the
-// epilogue (store / residual add / gated activation, optional RMS-norm scaling).  No CTA ever
-// waits for another.
+// by HBM bandwidth.  The grid is persistent (two CTAs per SM).  A CTA owns one K slice, keeps
+// that slice of X in shared memory for its whole life, and its warps walk over groups of R
+// weight rows with a register double buffer that keeps loads in flight across groups; warps
+// never synchronise with each other after the X slice is staged.  With more than one K slice
+// a warp leaves its fp32 partial sums in scratch and the warp that arrives last at the group's
+// ticket adds them in slice order (deterministic) and runs the epilogue (store / residual add /
+// gated activation, optional RMS-norm scaling).  Nothing ever waits for another CTA.  The first
+// weight loads are issued before the programmatic-dependent-launch wait, so they overlap the
+// tail of the kernel that produces X.
 #include "gemm.cuh"
 
 namespace csd {
@@ -15,44 +18,59 @@ namespace csd {
 constexpr int GT = 256;          // threads per CTA
 constexpr int GW = GT / 32;      // warps per CTA
 constexpr int KSTEP = 256;       // K elements one warp covers per step (32 lanes x 8 bf16)
+constexpr int CTAS_PER_SM = 2;
+constexpr size_t SMEM_BUDGET = 110 * 1024;   // per CTA, so that two CTAs share an SM
 
 template <int M, bool DUAL>
 struct RowsPerWarp {
-    static constexpr int value = DUAL ? (M <= 5 ? 4 : (M <= 9 ? 2 : 1)) : (M <= 9 ? 4 : 2);
+    static constexpr int value = DUAL ? (M <= 9 ? 2 : 1) : (M <= 9 ? 4 : 2);
 };
 
 struct LinearPlan {
-    int R, TN, ntiles, steps_total, steps_per, kslices, KSP;
-    size_t smem, unit_floats;
+    int R, NV, groups, steps_total, steps_per, kslices, KSP, grid;
+    size_t smem, scratch_floats;
 };
 
 static int rows_per_warp(int m, bool dual) {
-    return dual ? (m <= 5 ? 4 : (m <= 9 ? 2 : 1)) : (m <= 9 ? 4 : 2);
+    return dual ? (m <= 9 ? 2 : 1) : (m <= 9 ? 4 : 2);
+}
+
+static int sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
 }
 
 static LinearPlan plan_linear(int m, int N, int K, bool dual) {
     LinearPlan p;
     p.R = rows_per_warp(m, dual);
-    p.TN = GW * p.R;
-    p.ntiles = (N + p.TN - 1) / p.TN;
+    p.NV = (dual ? 2 : 1) * p.R * m;                       // partial sums one warp produces per row group
+    p.groups = (N + p.R - 1) / p.R;
     p.steps_total = (K + KSTEP - 1) / KSTEP;
-    int max_steps = (56 * 1024) / (m * KSTEP * 4);       // X slice of at most 56 KB
-    if (max_steps < 1) max_steps = 1;
-    int kslices = (p.steps_total + max_steps - 1) / max_steps;
-    const int want_units = 148 * 6;
-    int by_units = (want_units + p.ntiles - 1) / p.ntiles;
-    if (by_units > kslices) kslices = by_units;
-    int min_steps = 2;                                    // keep at least two steps per slice
-    int cap = p.steps_total / min_steps;
-    if (cap < 1) cap = 1;
-    if (kslices > cap) kslices = cap;
-    int need = (p.steps_total + max_steps - 1) / max_steps;
-    if (kslices < need) kslices = need;
+    const size_t red = (size_t)GW * p.NV * 33 * sizeof(float) + 64 * sizeof(float);
+    int kslices = 1;
+    for (;; ++kslices) {
+        int per = (p.steps_total + kslices - 1) / kslices;
+        if ((size_t)m * per * KSTEP * sizeof(float) + red <= SMEM_BUDGET || per == 1) break;
+    }
     p.steps_per = (p.steps_total + kslices - 1) / kslices;
     p.kslices = (p.steps_total + p.steps_per - 1) / p.steps_per;
     p.KSP = p.steps_per * KSTEP;
-    p.unit_floats = (size_t)(dual ? 2 : 1) * m * p.TN + m;
-    p.smem = ((size_t)m * p.KSP + (size_t)(dual ? 2 : 1) * m * p.TN + m + 8) * sizeof(float);
+    p.smem = (size_t)m * p.KSP * sizeof(float) + red;
+    // persistent grid: every SM gets CTAS_PER_SM CTAs, a multiple of the slice count, and no more
+    // warps per slice than there are row groups
+    int grid = sm_count() * CTAS_PER_SM;
+    int need = ((p.groups + GW - 1) / GW) * p.kslices;
+    if (grid > need) grid = need;
+    grid = (grid / p.kslices) * p.kslices;
+    if (grid < p.kslices) grid = p.kslices;
+    p.grid = grid;
+    p.scratch_floats = p.kslices > 1 ? (size_t)p.kslices * p.groups * p.NV + (size_t)p.kslices * m : 0;
     return p;
 }
 
@@ -65,7 +83,7 @@ struct GemmParams {
     float* partial;
     unsigned* tickets;
     int N, K, ldx, ldy, m;
-    int steps_per, kslices, KSP, ntiles;
+    int steps_per, kslices, KSP, groups;
     int epilogue;
     float eps;
 };
@@ -87,152 +105,188 @@ __device__ __forceinline__ float dot8(const uint4& w, const float4& a, const flo
     return acc;
 }
 
+// Programmatic dependent launch: the weights do not depend on the previous kernel, so a CTA may
+// start streaming them before the producer of X has finished; it must wait before reading X.
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 template <int M, bool DUAL>
-__global__ void __launch_bounds__(GT)
+__global__ void __launch_bounds__(GT, CTAS_PER_SM)
 skinny_gemm_kernel(const GemmParams p) {
     constexpr int R = RowsPerWarp<M, DUAL>::value;
-    constexpr int TN = GW * R;
     constexpr int NT = DUAL ? 2 : 1;
+    constexpr int NV = NT * R * M;               // sums one warp produces per row group
     extern __shared__ __align__(16) float smem[];
-    float* xs = smem;                           // [M][KSP], each 256-step stored as [half][lane][4]
-    float* tile = xs + (size_t)M * p.KSP;       // [NT][M][TN]
-    float* ss = tile + NT * M * TN;             // [M] sum of squares of this K slice
-    __shared__ int s_last;
+    float* xs = smem;                            // [M][KSP], each 256-step stored as [half][lane][4]
+    float* ss = xs + (size_t)M * p.KSP;          // [64] sum of squares per row over this K slice
+    float* red_all = ss + 64;                    // [GW][NV][33]
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
-    const int ntile = blockIdx.x / p.kslices, ks = blockIdx.x % p.kslices;
+    const int ks = blockIdx.x % p.kslices;
+    const int cta_in_slice = blockIdx.x / p.kslices, ctas_per_slice = gridDim.x / p.kslices;
     const int k0 = ks * p.KSP;
-    const int k1 = min(p.K, k0 + p.KSP);
-    const int kw = k1 - k0;
+    const int kw = min(p.K, k0 + p.KSP) - k0;
     const int steps = (kw + KSTEP - 1) / KSTEP;
+    const int gw = cta_in_slice * GW + warp, nw = ctas_per_slice * GW;
+    float* red = red_all + (size_t)warp * NV * 33;
 
-    // ---- stage the X slice (times the norm gain) into shared memory, permuted for
-    //      conflict-free 128-bit reads: k = s*256 + lane*8 + h*4 + i  ->  s*256 + h*128 + lane*4 + i
-    for (int idx = tid; idx < M * steps * KSTEP; idx += GT) {
-        const int r = idx / (steps * KSTEP), kk = idx % (steps * KSTEP);
-        float v = 0.f;
-        if (r < p.m && kk < kw) {
-            v = p.X[(size_t)r * p.ldx + k0 + kk];
-            if (p.gain) v *= __bfloat162float(p.gain[k0 + kk]);
+    // weight row pointers of a row group (rows past N are clamped: loaded, never stored)
+    const __nv_bfloat16* wrow[NT][R];
+    auto set_rows = [&](int g) {
+#pragma unroll
+        for (int rr = 0; rr < R; ++rr) {
+            int n = g * R + rr;
+            if (n >= p.N) n = p.N - 1;
+            wrow[0][rr] = p.W + (size_t)n * p.K + k0 + lane * 8;
+            if (DUAL) wrow[NT - 1][rr] = p.W2 + (size_t)n * p.K + k0 + lane * 8;
+        }
+    };
+    const uint4 zero4 = make_uint4(0, 0, 0, 0);
+    uint4 wcur[NT][R], wnext[NT][R];
+    int g = gw;
+    if (g < p.groups) {                          // first loads go out before the dependency wait
+        set_rows(g);
+#pragma unroll
+        for (int t = 0; t < NT; ++t)
+#pragma unroll
+            for (int rr = 0; rr < R; ++rr) wcur[t][rr] = (lane * 8 < kw) ? ldg_stream(wrow[t][rr]) : zero4;
+    }
+    grid_dependency_wait();
+    grid_launch_dependents();
+
+    // ---- stage the X slice (times the norm gain), permuted for conflict-free 128-bit reads:
+    //      k = s*256 + lane*8 + h*4 + i  ->  s*256 + h*128 + lane*4 + i
+    for (int idx = tid; idx < M * steps * (KSTEP / 4); idx += GT) {
+        const int r = idx / (steps * (KSTEP / 4)), q4 = idx % (steps * (KSTEP / 4));
+        const int kk = q4 * 4;
+        float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+        if (kk < kw) {                            // kw is a multiple of 8
+            v = *reinterpret_cast<const float4*>(p.X + (size_t)r * p.ldx + k0 + kk);
+            if (p.gain) {
+                const uint2 gb = *reinterpret_cast<const uint2*>(p.gain + k0 + kk);
+                v.x *= bf16lo(gb.x); v.y *= bf16hi(gb.x); v.z *= bf16lo(gb.y); v.w *= bf16hi(gb.y);
+            }
         }
         const int s = kk >> 8, o = kk & 255;
-        const int pos = (s << 8) + (((o >> 2) & 1) << 7) + ((o >> 3) << 2) + (o & 3);
-        xs[(size_t)r * p.KSP + pos] = v;
+        const int pos = (s << 8) + (((o >> 2) & 1) << 7) + ((o >> 3) << 2);
+        *reinterpret_cast<float4*>(xs + (size_t)r * p.KSP + pos) = v;
     }
     if (p.gain) {
         for (int r = warp; r < M; r += GW) {
             float a = 0.f;
-            if (r < p.m)
-                for (int kk = lane; kk < kw; kk += 32) {
-                    float v = p.X[(size_t)r * p.ldx + k0 + kk];
-                    a = fmaf(v, v, a);
-                }
+            for (int kk = lane * 4; kk < kw; kk += 128) {
+                const float4 v = *reinterpret_cast<const float4*>(p.X + (size_t)r * p.ldx + k0 + kk);
+                a = fmaf(v.x, v.x, a); a = fmaf(v.y, v.y, a); a = fmaf(v.z, v.z, a); a = fmaf(v.w, v.w, a);
+            }
             a = warp_sum(a);
             if (lane == 0) ss[r] = a;
         }
     }
     __syncthreads();
-
-    // ---- stream R weight rows per warp
-    const int n_base = ntile * TN + warp * R;
-    const __nv_bfloat16* wrow[NT][R];
-#pragma unroll
-    for (int rr = 0; rr < R; ++rr) {
-        int n = n_base + rr;
-        if (n >= p.N) n = p.N - 1;              // clamped rows are loaded but never stored
-        wrow[0][rr] = p.W + (size_t)n * p.K + k0 + lane * 8;
-        if (DUAL) wrow[NT - 1][rr] = p.W2 + (size_t)n * p.K + k0 + lane * 8;
+    float* ss_part = p.partial + (size_t)p.kslices * p.groups * NV;   // [kslices][M]
+    if (p.kslices > 1 && p.gain) {
+        if (tid < M) ss_part[ks * M + tid] = ss[tid];
+        __threadfence();
+        __syncthreads();
     }
-    float acc[NT][R][M];
-#pragma unroll
-    for (int t = 0; t < NT; ++t)
-#pragma unroll
-        for (int rr = 0; rr < R; ++rr)
-#pragma unroll
-            for (int r = 0; r < M; ++r) acc[t][rr][r] = 0.f;
 
-    uint4 wcur[NT][R], wnext[NT][R];
-    const uint4 zero4 = make_uint4(0, 0, 0, 0);
-#pragma unroll
-    for (int t = 0; t < NT; ++t)
-#pragma unroll
-        for (int rr = 0; rr < R; ++rr) wcur[t][rr] = (lane * 8 < kw) ? ldg_stream(wrow[t][rr]) : zero4;
-
-    for (int s = 0; s < steps; ++s) {
-        const int knext = (s + 1) * KSTEP + lane * 8;
+    for (; g < p.groups; g += nw) {
+        float acc[NT][R][M];
 #pragma unroll
         for (int t = 0; t < NT; ++t)
 #pragma unroll
             for (int rr = 0; rr < R; ++rr)
-                wnext[t][rr] = (s + 1 < steps && knext < kw) ? ldg_stream(wrow[t][rr] + (s + 1) * KSTEP) : zero4;
-        const float* xp = xs + (s << 8) + lane * 4;
 #pragma unroll
-        for (int r = 0; r < M; ++r) {
-            const float4 xa = *reinterpret_cast<const float4*>(xp + (size_t)r * p.KSP);
-            const float4 xb = *reinterpret_cast<const float4*>(xp + (size_t)r * p.KSP + 128);
+                for (int r = 0; r < M; ++r) acc[t][rr][r] = 0.f;
+        const int g_next = g + nw;
+        for (int s = 0; s < steps; ++s) {
+            // prefetch the next step, or the first step of this warp's next row group
+            if (s + 1 < steps) {
+                const bool ok = (s + 1) * KSTEP + lane * 8 < kw;
+#pragma unroll
+                for (int t = 0; t < NT; ++t)
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr)
+                        wnext[t][rr] = ok ? ldg_stream(wrow[t][rr] + (s + 1) * KSTEP) : zero4;
+            } else if (g_next < p.groups) {
+                set_rows(g_next);
+#pragma unroll
+                for (int t = 0; t < NT; ++t)
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr) wnext[t][rr] = (lane * 8 < kw) ? ldg_stream(wrow[t][rr]) : zero4;
+            }
+            const float* xp = xs + (s << 8) + lane * 4;
+#pragma unroll
+            for (int r = 0; r < M; ++r) {
+                const float4 xa = *reinterpret_cast<const float4*>(xp + (size_t)r * p.KSP);
+                const float4 xb = *reinterpret_cast<const float4*>(xp + (size_t)r * p.KSP + 128);
+#pragma unroll
+                for (int t = 0; t < NT; ++t)
+#pragma unroll
+                    for (int rr = 0; rr < R; ++rr) acc[t][rr][r] = dot8(wcur[t][rr], xa, xb, acc[t][rr][r]);
+            }
 #pragma unroll
             for (int t = 0; t < NT; ++t)
 #pragma unroll
-                for (int rr = 0; rr < R; ++rr) acc[t][rr][r] = dot8(wcur[t][rr], xa, xb, acc[t][rr][r]);
+                for (int rr = 0; rr < R; ++rr) wcur[t][rr] = wnext[t][rr];
         }
+        // ---- sum over lanes through shared memory: value v of lane l -> red[v][l]
+        __syncwarp();
 #pragma unroll
         for (int t = 0; t < NT; ++t)
 #pragma unroll
-            for (int rr = 0; rr < R; ++rr) wcur[t][rr] = wnext[t][rr];
-    }
-
-    // ---- reduce over lanes, gather the CTA's tile in shared memory
+            for (int rr = 0; rr < R; ++rr)
 #pragma unroll
-    for (int t = 0; t < NT; ++t)
+                for (int r = 0; r < M; ++r) red[((t * R + rr) * M + r) * 33 + lane] = acc[t][rr][r];
+        __syncwarp();
+        for (int v = lane; v < NV; v += 32) {
+            const float* row = red + v * 33;
+            float sum = 0.f;
 #pragma unroll
-        for (int rr = 0; rr < R; ++rr)
-#pragma unroll
-            for (int r = 0; r < M; ++r) {
-                float v = warp_sum(acc[t][rr][r]);
-                if (lane == 0) tile[(t * M + r) * TN + warp * R + rr] = v;
+            for (int j = 0; j < 32; ++j) sum += row[j];
+            red[v * 33 + 32] = sum;              // column 32 holds the finished sum
+        }
+        __syncwarp();
+        if (p.kslices > 1) {
+            float* mine = p.partial + ((size_t)ks * p.groups + g) * NV;
+            for (int v = lane; v < NV; v += 32) mine[v] = red[v * 33 + 32];
+            __threadfence();
+            __syncwarp();
+            unsigned old = 0;
+            if (lane == 0) old = atomicAdd(&p.tickets[g], 1u);
+            old = __shfl_sync(0xffffffffu, old, 0);
+            if (old != (unsigned)p.kslices - 1u) continue;     // another slice finishes this group
+            __threadfence();
+            for (int v = lane; v < NV; v += 32) {
+                float sum = 0.f;
+                for (int c = 0; c < p.kslices; ++c) sum += __ldcg(p.partial + ((size_t)c * p.groups + g) * NV + v);
+                red[v * 33 + 32] = sum;
             }
-    __syncthreads();
-
-    constexpr int UNIT = NT * M * TN;
-    if (p.kslices > 1) {
-        float* mine = p.partial + ((size_t)ntile * p.kslices + ks) * (UNIT + M);
-        for (int i = tid; i < UNIT; i += GT) mine[i] = tile[i];
-        if (p.gain && tid < M) mine[UNIT + tid] = ss[tid];
-        __threadfence();
-        __syncthreads();
-        if (tid == 0) {
-            unsigned old = atomicAdd(&p.tickets[ntile], 1u);
-            s_last = (old == (unsigned)p.kslices - 1u);
-            if (s_last) p.tickets[ntile] = 0u;     // ready for the next launch
+            if (lane == 0) p.tickets[g] = 0u;                  // ready for the next launch
+            __syncwarp();
         }
-        __syncthreads();
-        if (!s_last) return;
-        __threadfence();
-        const float* all = p.partial + (size_t)ntile * p.kslices * (UNIT + M);
-        for (int i = tid; i < UNIT + M; i += GT) {
-            if (i >= UNIT && !p.gain) break;
-            float v = 0.f;
-            for (int c = 0; c < p.kslices; ++c) v += __ldcg(all + (size_t)c * (UNIT + M) + i);
-            if (i < UNIT) tile[i] = v; else ss[i - UNIT] = v;
+        // ---- epilogue: lane handles (row of the group, block row)
+        for (int v = lane; v < R * M; v += 32) {
+            const int rr = v / M, r = v % M, n = g * R + rr;
+            if (n >= p.N) continue;
+            float scale = 1.f;
+            if (p.gain) {
+                float q = ss[r];
+                if (p.kslices > 1) {
+                    q = 0.f;
+                    for (int c = 0; c < p.kslices; ++c) q += __ldcg(ss_part + c * M + r);
+                }
+                scale = rsqrtf(q / (float)p.K + p.eps);
+            }
+            float val = red[v * 33 + 32] * scale;
+            if (DUAL) {
+                const float up = red[(R * M + v) * 33 + 32] * scale;
+                val = (p.epilogue == EPI_GEGLU ? gelu_tanh_f(val) : silu_f(val)) * up;
+            }
+            float* y = p.Y + (size_t)r * p.ldy + n;
+            if (p.epilogue == EPI_ADD) *y += val; else *y = val;
         }
-        __syncthreads();
-    }
-
-    // ---- epilogue
-    for (int i = tid; i < M * TN; i += GT) {
-        const int r = i / TN, c = i % TN;
-        const int n = ntile * TN + c;
-        if (r >= p.m || n >= p.N) continue;
-        float v = tile[r * TN + c];
-        float scale = 1.f;
-        if (p.gain) scale = rsqrtf(ss[r] / (float)p.K + p.eps);
-        v *= scale;
-        if (DUAL) {
-            float u = tile[(M + r) * TN + c] * scale;
-            v = (p.epilogue == EPI_GEGLU ? gelu_tanh_f(v) : silu_f(v)) * u;
-        }
-        float* y = p.Y + (size_t)r * p.ldy + n;
-        if (p.epilogue == EPI_ADD) *y += v; else *y = v;
+        __syncwarp();
     }
 }
 
@@ -241,12 +295,21 @@ static csd_status launch_one(const GemmParams& gp, const LinearPlan& pl, cudaStr
     auto kern = skinny_gemm_kernel<M, DUAL>;
     static bool attr_set = false;   // per instantiation
     if (!attr_set) {
-        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 100 * 1024));
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)SMEM_BUDGET + 4096));
         attr_set = true;
     }
-    kern<<<(unsigned)(pl.ntiles * pl.kslices), GT, pl.smem, st>>>(gp);
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)pl.grid);
+    cfg.blockDim = dim3(GT);
+    cfg.dynamicSmemBytes = pl.smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, gp));
     count_launch();
-    CSD_CUDA(cudaGetLastError());
     return CSD_OK;
 }
 
@@ -254,13 +317,13 @@ size_t linear_scratch_bytes(int m, int N, int K, bool dual) {
     size_t worst = 0;
     for (int mm = 1; mm <= m; ++mm) {
         LinearPlan pl = plan_linear(mm, N, K, dual);
-        size_t b = pl.kslices > 1 ? (size_t)pl.ntiles * pl.kslices * pl.unit_floats * sizeof(float) : 0;
+        size_t b = pl.scratch_floats * sizeof(float);
         if (b > worst) worst = b;
     }
     return align_up(worst, 256);
 }
 
-int linear_ticket_count(int N) { return (N + GW - 1) / GW + 1; }   // TN >= GW columns per tile
+int linear_ticket_count(int N) { return N + 1; }   // one ticket per row group, at least one row each
 
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     if (!a.W || !a.X || !a.Y || a.m < 1 || a.m > CSD_MAX_ROWS || a.N < 1 || a.K < 8 || (a.K & 7))
@@ -273,7 +336,7 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     GemmParams gp;
     gp.W = a.W; gp.W2 = a.W2; gp.X = a.X; gp.gain = a.gain; gp.Y = a.Y; gp.partial = a.partial;
     gp.tickets = a.tickets; gp.N = a.N; gp.K = a.K; gp.ldx = a.ldx; gp.ldy = a.ldy; gp.m = a.m;
-    gp.steps_per = pl.steps_per; gp.kslices = pl.kslices; gp.KSP = pl.KSP; gp.ntiles = pl.ntiles;
+    gp.steps_per = pl.steps_per; gp.kslices = pl.kslices; gp.KSP = pl.KSP; gp.groups = pl.groups;
     gp.epilogue = a.epilogue; gp.eps = a.eps;
 #define CSD_CASE(MM)                                                              \
     case MM:                                                                      \

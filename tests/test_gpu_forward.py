@@ -92,7 +92,7 @@ def test_encoder_decoder(b, orc):
     pos = 0
     for m in (1, 17, 5, 17):
         got = gm.csd_review_forward(to_dev_i32(dec[pos:pos + m]), pos).cpu().numpy()
-        assert rel_l2(got, om.review_forward(dec[pos:pos + m], pos)) < 1e-3
+        assert rel_l2(got, om.review_forward(dec[pos:pos + m], pos)) < 2e-3
         pos += m
 
 
