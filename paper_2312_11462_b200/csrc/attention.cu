@@ -123,9 +123,9 @@ block_attention_kernel(const AttnParams p) {
             const float nm = fmaxf(old, tmax);
             float p0 = 0.f, p1 = 0.f, alpha = 1.f;
             if (nm > -INFINITY) {
-                p0 = __expf(s0 - nm);
-                p1 = __expf(s1 - nm);
-                alpha = __expf(old - nm);
+                p0 = expf(s0 - nm);
+                p1 = expf(s1 - nm);
+                alpha = expf(old - nm);
             }
             sc[r * TILE + lane] = p0;
             sc[r * TILE + lane + 32] = p1;
@@ -209,7 +209,7 @@ block_attention_kernel(const AttnParams p) {
             const float* rec = all + ((size_t)s * MAXM + r) * REC;
             const float ms = __ldcg(rec + DH);
             if (ms > -INFINITY) {
-                const float w = __expf(ms - M);
+                const float w = expf(ms - M);
                 num = fmaf(__ldcg(rec + d), w, num);
                 den = fmaf(__ldcg(rec + DH + 1), w, den);
             }

@@ -11,7 +11,7 @@
 // gated activation, optional RMS-norm scaling).  Nothing ever waits for another CTA.  The first
 // weight loads are issued before the programmatic-dependent-launch wait, so they overlap the
 // tail of the kernel that produces X.
-#include "gemm.cuh"
+#include "gemm_tc.cuh"
 
 namespace csd {
 
@@ -19,6 +19,7 @@ constexpr int GT = 256;          // threads per CTA
 constexpr int GW = GT / 32;      // warps per CTA
 constexpr int KSTEP = 256;       // K elements one warp covers per step (32 lanes x 8 bf16)
 constexpr int CTAS_PER_SM = 2;
+constexpr int AUTO_TC_MIN_ROWS = 17;     // automatic choice: rows above this go to the tensor-core kernel
 constexpr size_t SMEM_BUDGET = 110 * 1024;   // per CTA, so that two CTAs share an SM
 
 template <int M, bool DUAL>
@@ -91,7 +92,7 @@ struct GemmParams {
 __device__ __forceinline__ float gelu_tanh_f(float x) {
     return 0.5f * x * (1.f + tanhf(0.7978845608028654f * (x + 0.044715f * x * x * x)));
 }
-__device__ __forceinline__ float silu_f(float x) { return x / (1.f + __expf(-x)); }
+__device__ __forceinline__ float silu_f(float x) { return x / (1.f + expf(-x)); }
 
 __device__ __forceinline__ float dot8(const uint4& w, const float4& a, const float4& b, float acc) {
     acc = fmaf(bf16lo(w.x), a.x, acc);
@@ -276,7 +277,7 @@ skinny_gemm_kernel(const GemmParams p) {
                     q = 0.f;
                     for (int c = 0; c < p.kslices; ++c) q += __ldcg(ss_part + c * M + r);
                 }
-                scale = rsqrtf(q / (float)p.K + p.eps);
+                scale = 1.f / sqrtf(q / (float)p.K + p.eps);
             }
             float val = red[v * 33 + 32] * scale;
             if (DUAL) {
@@ -320,6 +321,8 @@ size_t linear_scratch_bytes(int m, int N, int K, bool dual) {
         size_t b = pl.scratch_floats * sizeof(float);
         if (b > worst) worst = b;
     }
+    const size_t tc = tc_scratch_bytes(m, N, K, dual);
+    if (tc > worst) worst = tc;
     return align_up(worst, 256);
 }
 
@@ -331,6 +334,12 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     const bool dual = a.W2 != nullptr;
     if (dual != (a.epilogue == EPI_SWIGLU || a.epilogue == EPI_GEGLU)) return CSD_ERR_INVALID_ARG;
     if ((((uintptr_t)a.W) & 15) || (dual && (((uintptr_t)a.W2) & 15))) return CSD_ERR_INVALID_ARG;
+    if ((((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
+    // kernel choice: the tensor-core kernel wherever it applies when selected (or, on automatic,
+    // for blocks of more than AUTO_TC_MIN_ROWS rows, where the CUDA-core kernel is ALU-bound)
+    const int path = gemm_path();
+    if (path != 1 && tc_supported(a.m, a.N, a.K, dual) && (path == 2 || a.m > AUTO_TC_MIN_ROWS))
+        return launch_linear_tc(a, st);
     const LinearPlan pl = plan_linear(a.m, a.N, a.K, dual);
     if (pl.kslices > 1 && (!a.partial || !a.tickets)) return CSD_ERR_INVALID_ARG;
     GemmParams gp;
@@ -353,6 +362,12 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
 }  // namespace csd
 
 using namespace csd;
+
+extern "C" csd_status csd_set_gemm_path(int path) {
+    if (path < 0 || path > 2) return CSD_ERR_INVALID_ARG;
+    set_gemm_path(path);
+    return CSD_OK;
+}
 
 extern "C" size_t csd_linear_workspace_bytes(int m, int N, int K) {
     if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8) return 0;
