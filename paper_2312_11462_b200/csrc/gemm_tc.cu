@@ -71,7 +71,11 @@ static TcPlan tc_plan(int m, int N, int K, bool dual) {
         if (ctas_per_slice < 1) continue;
         if (ctas_per_slice > tiles) ctas_per_slice = tiles;
         const int rounds = (tiles + ctas_per_slice - 1) / ctas_per_slice;
-        const double cost = (double)rounds * (per + 1.5) + (ks > 1 ? 1.0 : 0.0) + 8.0 / stages;
+        // time in units of one k-block streamed by one SM: the slice of every tile, an accumulator
+        // read-out per tile, the split of this slice of X (exposed before the first MMA), and a
+        // penalty when the ring is too shallow to cover the memory latency
+        double cost = (double)rounds * (per + 1.5) + 0.06 * m * per + (ks > 1 ? 1.0 : 0.0);
+        if (stages < 6) cost *= 1.0 + 0.25 * (6 - stages);
         if (cost < best_cost) {
             best_cost = cost;
             best.npad = npad; best.tiles = tiles; best.kblocks = kblocks; best.kb_per = per; best.kslices = ks;
@@ -221,7 +225,6 @@ struct __align__(8) TcCtrl {
     uint32_t tmem_base;
     int abort_flag, last_flag;
     float ss[32];
-    float ss_warp[32 * 6];
 };
 
 __device__ __forceinline__ float tc_gelu(float x) {
@@ -292,52 +295,62 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     __syncthreads();
     {
         const int chunks = kw / 8;                         // 16-byte chunks per row (K is a multiple of 8)
-        for (int r = 0; r < M; ++r) {
+        for (int r = warp; r < M; r += TC_THREADS / 32) {  // one warp per row, four chunks in flight per lane
             float sq = 0.f;
-            for (int c = tid; c < chunks; c += TC_THREADS) {
-                const float* src = p.X + (size_t)r * p.ldx + k0 + c * 8;
-                const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
-                float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+            for (int c0 = lane; c0 < chunks; c0 += 128) {
+                float4 xa[4], xb[4];
+                uint4 gg[4];
 #pragma unroll
-                for (int e = 0; e < 8; ++e) sq = fmaf(v[e], v[e], sq);
-                if (p.gain) {
-                    const uint4 g = *reinterpret_cast<const uint4*>(p.gain + k0 + c * 8);
-                    v[0] *= bf16lo(g.x); v[1] *= bf16hi(g.x); v[2] *= bf16lo(g.y); v[3] *= bf16hi(g.y);
-                    v[4] *= bf16lo(g.z); v[5] *= bf16hi(g.z); v[6] *= bf16lo(g.w); v[7] *= bf16hi(g.w);
-                }
-                uint32_t t1[4], t2[4], t3[4];
-#pragma unroll
-                for (int e = 0; e < 8; e += 2) {
-                    uint32_t w1 = 0, w2 = 0, w3 = 0;
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const float x = v[e + h];
-                        const uint16_t b1 = float_to_bf16_bits(x);
-                        const float r1 = x - bf16_bits_to_float(b1);
-                        const uint16_t b2 = float_to_bf16_bits(r1);
-                        const uint16_t b3 = float_to_bf16_bits(r1 - bf16_bits_to_float(b2));
-                        w1 |= (uint32_t)b1 << (16 * h); w2 |= (uint32_t)b2 << (16 * h); w3 |= (uint32_t)b3 << (16 * h);
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + 32 * u;
+                    if (c < chunks) {
+                        const float* src = p.X + (size_t)r * p.ldx + k0 + c * 8;
+                        xa[u] = *reinterpret_cast<const float4*>(src);
+                        xb[u] = *reinterpret_cast<const float4*>(src + 4);
+                        if (p.gain) gg[u] = *reinterpret_cast<const uint4*>(p.gain + k0 + c * 8);
                     }
-                    t1[e / 2] = w1; t2[e / 2] = w2; t3[e / 2] = w3;
                 }
-                const int kb = c >> 3, cc = c & 7;
-                unsigned char* blk = xs + (size_t)kb * NPAD * 128;
-                const int j1 = r, j2 = M + r, j3 = 2 * M + r;
-                *reinterpret_cast<uint4*>(blk + j1 * 128 + ((cc ^ (j1 & 7)) << 4)) = make_uint4(t1[0], t1[1], t1[2], t1[3]);
-                *reinterpret_cast<uint4*>(blk + j2 * 128 + ((cc ^ (j2 & 7)) << 4)) = make_uint4(t2[0], t2[1], t2[2], t2[3]);
-                *reinterpret_cast<uint4*>(blk + j3 * 128 + ((cc ^ (j3 & 7)) << 4)) = make_uint4(t3[0], t3[1], t3[2], t3[3]);
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int c = c0 + 32 * u;
+                    if (c >= chunks) continue;
+                    float v[8] = {xa[u].x, xa[u].y, xa[u].z, xa[u].w, xb[u].x, xb[u].y, xb[u].z, xb[u].w};
+#pragma unroll
+                    for (int e = 0; e < 8; ++e) sq = fmaf(v[e], v[e], sq);
+                    if (p.gain) {
+                        const uint4 g = gg[u];
+                        v[0] *= bf16lo(g.x); v[1] *= bf16hi(g.x); v[2] *= bf16lo(g.y); v[3] *= bf16hi(g.y);
+                        v[4] *= bf16lo(g.z); v[5] *= bf16hi(g.z); v[6] *= bf16lo(g.w); v[7] *= bf16hi(g.w);
+                    }
+                    uint32_t t1[4], t2[4], t3[4];
+#pragma unroll
+                    for (int e = 0; e < 8; e += 2) {
+                        uint32_t w1 = 0, w2 = 0, w3 = 0;
+#pragma unroll
+                        for (int h = 0; h < 2; ++h) {
+                            const float x = v[e + h];
+                            const uint16_t b1 = float_to_bf16_bits(x);
+                            const float r1 = x - bf16_bits_to_float(b1);
+                            const uint16_t b2 = float_to_bf16_bits(r1);
+                            const uint16_t b3 = float_to_bf16_bits(r1 - bf16_bits_to_float(b2));
+                            w1 |= (uint32_t)b1 << (16 * h); w2 |= (uint32_t)b2 << (16 * h); w3 |= (uint32_t)b3 << (16 * h);
+                        }
+                        t1[e / 2] = w1; t2[e / 2] = w2; t3[e / 2] = w3;
+                    }
+                    const int kb = c >> 3, cc = c & 7;
+                    unsigned char* blk = xs + (size_t)kb * NPAD * 128;
+                    const int j1 = r, j2 = M + r, j3 = 2 * M + r;
+                    *reinterpret_cast<uint4*>(blk + j1 * 128 + ((cc ^ (j1 & 7)) << 4)) = make_uint4(t1[0], t1[1], t1[2], t1[3]);
+                    *reinterpret_cast<uint4*>(blk + j2 * 128 + ((cc ^ (j2 & 7)) << 4)) = make_uint4(t2[0], t2[1], t2[2], t2[3]);
+                    *reinterpret_cast<uint4*>(blk + j3 * 128 + ((cc ^ (j3 & 7)) << 4)) = make_uint4(t3[0], t3[1], t3[2], t3[3]);
+                }
             }
             sq = warp_sum(sq);
-            if (lane == 0) ctl->ss_warp[r * 6 + warp] = sq;
+            if (lane == 0) ctl->ss[r] = sq;
         }
     }
     fence_async_smem();
     __syncthreads();
-    if (tid < M) {
-        float q = 0.f;
-        for (int w = 0; w < 6; ++w) q += ctl->ss_warp[tid * 6 + w];
-        ctl->ss[tid] = q;
-    }
     float* ss_part = p.partial + (size_t)p.kslices * p.tiles * TILE_N * M * NT;   // [kslices][M]
     __syncthreads();
     if (p.kslices > 1 && p.gain) {
