@@ -174,6 +174,30 @@ csd_status csd_spec_accept(const float* target_logits_dev, const float* draft_lo
                            int32_t* n_accepted_dev, int32_t* out_token_dev, void* workspace_dev,
                            size_t workspace_bytes, void* stream);
 
+/* The same review rule for callers that cannot allocate device memory (the paper has no
+ * counterpart; this is a deployment convenience).  Some hosts of this library run where
+ * cudaMalloc is off limits: inside a real-time serving loop that forbids allocator calls after
+ * start-up, inside a process whose memory budget is fixed by another component, or from code
+ * that only holds the buffers it was handed.  csd_spec_accept_static needs no workspace argument:
+ * its scratch is a fixed 2 MiB array that is part of the library image (every GPU that loads the
+ * library carries it until the process exits; csd_spec_accept_static_capacity returns the size).
+ * The call allocates nothing, on the host or on the device, and takes the same inputs and gives
+ * the same outputs as csd_spec_accept.  Differences:
+ *   - problems whose scratch need (csd_spec_accept_workspace_bytes) exceeds the capacity are
+ *     refused with CSD_ERR_CAPACITY; 64 rows x 16 drafted tokens x 128256 logits fits;
+ *   - a token id outside [0, V) is still treated as rejected, but is not recorded in the device
+ *     status word (recording would need that word to exist, and creating it allocates);
+ *   - the first call on each device looks up the device address of the array (with that device
+ *     current); make that first call outside any stream capture;
+ *   - all calls share the one array, which keeps whatever the previous call left in it.  Nothing
+ *     in it has to start at zero, but two calls that overlap on the GPU (different streams) would
+ *     overwrite each other's intermediate results: issue them on one stream, or order them. */
+size_t csd_spec_accept_static_capacity(void);
+csd_status csd_spec_accept_static(const float* target_logits_dev, const float* draft_logits_dev,
+                                  const int32_t* onehot_dev, const int32_t* draft_tokens_dev, int rows, int k, int V,
+                                  float temperature, float lenience, uint64_t seed, uint64_t step,
+                                  int32_t* n_accepted_dev, int32_t* out_token_dev, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Max-Gram statistical drafter (Section 3.3, Appendix A): the longest suffix of the sequence
  * (at most max_order tokens) that occurs in the haystack followed by at least one haystack

@@ -85,6 +85,8 @@ lib.csd_linear.argtypes = [_vp, _i, _i, _vp, _i, _vp, _vp, _sz, _vp]
 lib.csd_spec_accept_workspace_bytes.restype = _sz
 lib.csd_spec_accept_workspace_bytes.argtypes = [_i, _i, _i]
 lib.csd_spec_accept.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp, _sz, _vp]
+lib.csd_spec_accept_static_capacity.restype = _sz
+lib.csd_spec_accept_static.argtypes = [_vp, _vp, _vp, _vp, _i, _i, _i, _f, _f, _u64, _u64, _vp, _vp, _vp]
 lib.csd_mag_workspace_bytes.restype = _sz
 lib.csd_mag_workspace_bytes.argtypes = [_i, _i, _i]
 lib.csd_mag_create.argtypes = [_vp, _i, _i, _vp, _i, _i, _vp, _sz, _vp, _vp]
@@ -233,6 +235,20 @@ def csd_spec_accept(target_logits: torch.Tensor, draft_logits: Optional[torch.Te
            lib.csd_spec_accept(_ptr(target_logits), _ptr(draft_logits), _ptr(onehot), _ptr(draft_tokens), rows, k, V,
                                temperature, lenience, seed, step, _ptr(out[0]), _ptr(out[1]), _ptr(workspace),
                                workspace.numel(), _stream()))
+    return out
+
+
+def csd_spec_accept_static(target_logits: torch.Tensor, draft_logits: Optional[torch.Tensor],
+                           draft_tokens: torch.Tensor, temperature: float, lenience: float = 1.0, seed: int = 0,
+                           step: int = 0, onehot: Optional[torch.Tensor] = None, out: Sequence[torch.Tensor] = None):
+    """The review rule through the entry point that allocates nothing: the caller supplies every
+    buffer, outputs included (`out` = (n_accepted, out_token), int32 [rows] each)."""
+    rows, k1, V = target_logits.shape
+    assert out is not None and out[0].dtype == torch.int32 and out[1].dtype == torch.int32
+    _check("csd_spec_accept_static",
+           lib.csd_spec_accept_static(_ptr(target_logits), _ptr(draft_logits), _ptr(onehot), _ptr(draft_tokens), rows,
+                                      k1 - 1, V, temperature, lenience, seed, step, _ptr(out[0]), _ptr(out[1]),
+                                      _stream()))
     return out
 
 

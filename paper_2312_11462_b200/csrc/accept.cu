@@ -9,6 +9,7 @@
 //           that the chosen token does not depend on the summation order.
 #include "common.cuh"
 #include "philox.cuh"
+#include <mutex>
 
 namespace csd {
 
@@ -440,6 +441,84 @@ extern "C" csd_status csd_spec_accept(const float* target_logits_dev, const floa
     accept_decide_kernel<<<rows, 128, 0, st>>>(target_logits_dev, dl, onehot_dev, draft_tokens_dev, rows, k, V,
                                                temperature, lenience, seed, step, part, L.nchunk_a,
                                                n_accepted_dev, out_token_dev, info, status);
+    count_launch(2);
+    if (!greedy) {
+        dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
+        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, L.nchunk_r);
+        resample_mass_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart, L.nchunk_r);
+        resample_pick_kernel<<<rows, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart,
+                                                          L.nchunk_r, out_token_dev);
+        count_launch(3);
+    }
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Variant for callers that must not allocate: its scratch is a fixed array inside the library.
+// ---------------------------------------------------------------------------------------------
+namespace csd {
+constexpr size_t STATIC_SCRATCH_BYTES = (size_t)2 << 20;   // 2 MiB, held by every GPU that loads the library
+static __device__ __align__(256) unsigned char g_accept_scratch[STATIC_SCRATCH_BYTES];
+constexpr int MAX_DEVICES = 64;
+static void* g_accept_scratch_ptr[MAX_DEVICES];             // device address of the array, per device
+static std::mutex g_accept_scratch_mu;
+}  // namespace csd
+
+extern "C" size_t csd_spec_accept_static_capacity(void) { return STATIC_SCRATCH_BYTES; }
+
+extern "C" csd_status csd_spec_accept_static(const float* target_logits_dev, const float* draft_logits_dev,
+                                             const int32_t* onehot_dev, const int32_t* draft_tokens_dev, int rows,
+                                             int k, int V, float temperature, float lenience, uint64_t seed,
+                                             uint64_t step, int32_t* n_accepted_dev, int32_t* out_token_dev,
+                                             void* stream) {
+    if (rows < 0 || k < 0 || k > MAX_K || V < 1 || !(temperature >= 0.f) || !(lenience >= 1.f))
+        return CSD_ERR_INVALID_ARG;
+    if (rows == 0) return CSD_OK;
+    if (!target_logits_dev || !n_accepted_dev || !out_token_dev) return CSD_ERR_INVALID_ARG;
+    if (k > 0 && !draft_tokens_dev) return CSD_ERR_INVALID_ARG;
+    const AcceptLayout L = accept_layout(rows, k, V);
+    if (L.total > STATIC_SCRATCH_BYTES) return CSD_ERR_CAPACITY;   // the problem does not fit the fixed scratch
+    if (L.nchunk_a > 65535 || L.nchunk_r > 65535) return CSD_ERR_UNSUPPORTED;
+    // Set-up, once per device: in host code the array's name is only a handle, so ask the runtime
+    // for the address the kernels can use.  Nothing is allocated here.
+    int dev = 0;
+    CSD_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= MAX_DEVICES) return CSD_ERR_UNSUPPORTED;
+    char* ws = nullptr;
+    {
+        std::lock_guard<std::mutex> lk(g_accept_scratch_mu);
+        if (!g_accept_scratch_ptr[dev]) {
+            void* p = nullptr;
+            CSD_CUDA(cudaGetSymbolAddress(&p, g_accept_scratch));
+            g_accept_scratch_ptr[dev] = p;
+        }
+        ws = (char*)g_accept_scratch_ptr[dev];
+    }
+    cudaStream_t st = (cudaStream_t)stream;
+    StatPartial* part = (StatPartial*)(ws + L.part_off);
+    RowInfo* info = (RowInfo*)(ws + L.info_off);
+    double2* zpart = (double2*)(ws + L.z_off);
+    double* rpart = (double*)(ws + L.r_off);
+    const bool greedy = temperature == 0.f;
+    const float invT = greedy ? 1.f : 1.f / temperature;
+    const bool use_d = draft_logits_dev != nullptr && k > 0 && !greedy;
+    const float* dl = use_d ? draft_logits_dev : nullptr;
+    const long long n_tvec = (long long)rows * (k + 1);
+    const long long nvec = n_tvec + (use_d ? (long long)rows * k : 0);
+    if (nvec > 0x7fffffffLL) return CSD_ERR_UNSUPPORTED;
+    const bool vec_ok = (V % 4 == 0) && (((uintptr_t)target_logits_dev & 15) == 0) &&
+                        (!use_d || ((uintptr_t)draft_logits_dev & 15) == 0);
+    // Every word of the scratch that a pass reads is written by an earlier pass of the same call,
+    // so nothing has to be cleared even though the array still holds the previous call's data.
+    dim3 grid((unsigned)nvec, (unsigned)L.nchunk_a);
+    if (vec_ok)
+        accept_stats_kernel<true><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
+    else
+        accept_stats_kernel<false><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
+    accept_decide_kernel<<<rows, 128, 0, st>>>(target_logits_dev, dl, onehot_dev, draft_tokens_dev, rows, k, V,
+                                               temperature, lenience, seed, step, part, L.nchunk_a,
+                                               n_accepted_dev, out_token_dev, info, nullptr);
     count_launch(2);
     if (!greedy) {
         dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
