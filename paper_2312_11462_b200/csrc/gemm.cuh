@@ -19,7 +19,20 @@ struct LinearArgs {
     int epilogue = EPI_STORE;
     float* partial = nullptr;            // split-K scratch (linear_scratch_bytes)
     unsigned* tickets = nullptr;         // zero-initialised, linear_ticket_count entries
+    // ---- tensor-core path only: the block's rows as three bf16 terms x = b1 + b2 + b3
+    __nv_bfloat16* xs = nullptr;         // [3m][K] row-major, row = term * m + r
+    bool xs_ready = false;               // false: launch_linear splits X (times gain) into xs first
+    float* ssq = nullptr;                // [ssq_cnt][m] pieces of the sums of squares of the rows of X (gain != null)
+    int ssq_cnt = 0;                     // entries valid in ssq when xs_ready
+    // optional extra outputs for the GEMM that consumes Y next
+    __nv_bfloat16* out_xs = nullptr;     // three-term split of (Y * out_gain), [3m][out_ld]
+    int out_ld = 0;
+    const __nv_bfloat16* out_gain = nullptr;
+    float* out_ssq = nullptr;            // [4 * ceil(N/128)][m] pieces of the sums of squares of the rows of Y
 };
+
+int split_rows(int m);                   // 16, 32, 48 or 64 operand rows hold the 3m terms
+int split_ssq_entries(int K);            // ssq pieces the stand-alone split kernel writes
 
 size_t linear_scratch_bytes(int m, int N, int K, bool dual);
 int linear_ticket_count(int N);
