@@ -331,3 +331,83 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             }
         }
     } else {
+        // ---- epilogue warps: quadrant q of tensor memory holds weight rows q*32 .. q*32+31 of the tile
+        const int q = warp & 3, et = (warp - 2) * 32 + lane;
+        asm volatile("griddepcontrol.wait;" ::: "memory");
+        if (p.ssq_in && et < M) {               // rms-norm factor of every row from the pieces of its sum of squares
+            float sq = 0.f;
+            for (int c = 0; c < p.ssq_cnt; ++c) sq += __ldcg(p.ssq_in + (size_t)c * M + et);
+            ctl->scale[et] = 1.f / sqrtf(sq / (float)p.K + p.eps);
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        float* my_part = p.partial + (size_t)cta * 2 * NT * M * TILE_N;
+        int i = 0;
+        for (int seg = 0; i < items; ++seg) {
+            const int b = seg & 1;
+            const int tile = (int)((u0 + i) / p.nkb), kb_begin = (int)((u0 + i) % p.nkb);
+            const int seg_len = min(p.nkb - kb_begin, items - i);
+            i += seg_len;
+            if (!mbar_wait(&ctl->acc_full[b], (seg >> 1) & 1)) { *abort_flag = 1; break; }   // same outcome in all four warps
+            tc_fence_after();
+            const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * ACC_COLS);
+            float sums[NT][M];
+#pragma unroll
+            for (int u = 0; u < NT; ++u) {
+                float third[M], second[M];
+#pragma unroll
+                for (int r = 0; r < M; ++r) { sums[u][r] = 0.f; second[r] = 0.f; third[r] = 0.f; }
+#pragma unroll
+                for (int c0 = 0; c0 < NPAD; c0 += 16) {
+                    if (c0 >= 3 * M) break;
+                    float v[16];
+                    tc_ld16(taddr + (uint32_t)(u * NPAD + c0), v);
+#pragma unroll
+                    for (int c = 0; c < 16; ++c) {
+                        const int col = c0 + c;
+                        if (col < M) sums[u][col] = v[c];
+                        else if (col < 2 * M) second[col - M] = v[c];
+                        else if (col < 3 * M) third[col - 2 * M] = v[c];
+                    }
+                }
+#pragma unroll
+                for (int r = 0; r < M; ++r) sums[u][r] += second[r] + third[r];   // small terms first
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&ctl->acc_empty[b]);
+            const int col = q * 32 + lane, n = tile * TILE_N + col;
+            if (seg_len < p.nkb) {
+                // part of a tile: leave it in this CTA's slot (0 = the CTA's first segment, 1 = a later
+                // one); the CTA that arrives last adds all parts in CTA order and finishes the tile
+                float* mine = my_part + (size_t)(seg == 0 ? 0 : 1) * NT * M * TILE_N;
+#pragma unroll
+                for (int u = 0; u < NT; ++u)
+#pragma unroll
+                    for (int r = 0; r < M; ++r) mine[(u * M + r) * TILE_N + col] = sums[u][r];
+                __threadfence();
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int c_lo = cta_of_unit((long long)tile * p.nkb, units, ctas);
+                const int c_hi = cta_of_unit((long long)(tile + 1) * p.nkb - 1, units, ctas);
+                if (et == 0) {
+                    const unsigned old = atomicAdd(&p.tickets[tile], 1u);
+                    ctl->last_flag = (old == (unsigned)(c_hi - c_lo));
+                    if (ctl->last_flag) p.tickets[tile] = 0u;
+                }
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int last = ctl->last_flag;
+                asm volatile("bar.sync 1, 128;" ::: "memory");
+                if (!last) continue;
+                __threadfence();
+#pragma unroll
+                for (int u = 0; u < NT; ++u)
+#pragma unroll
+                    for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
+                for (int c = c_lo; c <= c_hi; ++c) {
+                    const int slot = (int)(unit_begin(c, units, ctas) / p.nkb) == tile ? 0 : 1;
+                    const float* src = p.partial + ((size_t)c * 2 + slot) * NT * M * TILE_N + col;
+#pragma unroll
+                    for (int u = 0; u < NT; ++u)
+#pragma unroll
+                        for (int r = 0; r < M; ++r) sums[u][r] += __ldcg(src + (u * M + r) * TILE_N);
+                }
+            }
