@@ -411,3 +411,98 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                         for (int r = 0; r < M; ++r) sums[u][r] += __ldcg(src + (u * M + r) * TILE_N);
                 }
             }
+            // ---- finish the tile: this thread owns output column n for all M rows
+            float outv[M];
+#pragma unroll
+            for (int r = 0; r < M; ++r) {
+                const float scale = p.ssq_in ? ctl->scale[r] : 1.f;
+                float val = sums[0][r] * scale;
+                if (DUAL) {
+                    const float up = sums[NT - 1][r] * scale;
+                    val = (p.epilogue == EPI_GEGLU ? tc_gelu(val) : tc_silu(val)) * up;
+                }
+                if (n < p.N) {
+                    float* y = p.Y + (size_t)r * p.ldy + n;
+                    if (p.epilogue == EPI_ADD) val += *y;
+                    *y = val;
+                } else {
+                    val = 0.f;
+                }
+                outv[r] = val;
+            }
+            if (p.out_ssq) {                      // pieces of the rows' sums of squares, one per 32 columns
+#pragma unroll
+                for (int r = 0; r < M; ++r) {
+                    const float sq = warp_sum(outv[r] * outv[r]);
+                    if (lane == 0) p.out_ssq[(size_t)(tile * 4 + q) * M + r] = sq;
+                }
+            }
+            if (p.out_xs && n < p.N) {            // the rows as three bf16 terms for the GEMM that reads them next
+                const float g = p.out_gain ? __bfloat162float(p.out_gain[n]) : 1.f;
+#pragma unroll
+                for (int r = 0; r < M; ++r) {
+                    uint16_t b1, b2, b3;
+                    split3(outv[r] * g, b1, b2, b3);
+                    uint16_t* o = reinterpret_cast<uint16_t*>(p.out_xs) + n;
+                    o[(size_t)r * p.out_ld] = b1;
+                    o[(size_t)(M + r) * p.out_ld] = b2;
+                    o[(size_t)(2 * M + r) * p.out_ld] = b3;
+                }
+            }
+        }
+    }
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    if (*abort_flag) {
+        if (tid == 0) set_status(p.status, CSD_ERR_TIMEOUT);
+        __nanosleep(2000000);          // let copies already in flight land before the CTA's memory is released
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
+
+// Stand-alone split of fp32 rows (times an optional gain) into three bf16 terms, plus the pieces of
+// each row's sum of squares.  grid = (K / 1024 rounded up, m).
+__global__ void __launch_bounds__(128)
+split_rows_kernel(const float* __restrict__ X, int ldx, int K, int m, const __nv_bfloat16* __restrict__ gain,
+                  __nv_bfloat16* __restrict__ xs, float* __restrict__ ssq) {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const int r = blockIdx.y, k = (blockIdx.x * 128 + threadIdx.x) * 8;
+    float sq = 0.f;
+    if (k < K) {
+        const float* src = X + (size_t)r * ldx + k;
+        const float4 a = *reinterpret_cast<const float4*>(src), b = *reinterpret_cast<const float4*>(src + 4);
+        float v[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
+#pragma unroll
+        for (int e = 0; e < 8; ++e) sq = fmaf(v[e], v[e], sq);
+        if (gain) {
+            const uint4 g = *reinterpret_cast<const uint4*>(gain + k);
+            v[0] *= bf16lo(g.x); v[1] *= bf16hi(g.x); v[2] *= bf16lo(g.y); v[3] *= bf16hi(g.y);
+            v[4] *= bf16lo(g.z); v[5] *= bf16hi(g.z); v[6] *= bf16lo(g.w); v[7] *= bf16hi(g.w);
+        }
+        uint32_t t[3][4];
+#pragma unroll
+        for (int e = 0; e < 8; e += 2) {
+            uint16_t a1, a2, a3, c1, c2, c3;
+            split3(v[e], a1, a2, a3);
+            split3(v[e + 1], c1, c2, c3);
+            t[0][e / 2] = a1 | ((uint32_t)c1 << 16); t[1][e / 2] = a2 | ((uint32_t)c2 << 16);
+            t[2][e / 2] = a3 | ((uint32_t)c3 << 16);
+        }
+#pragma unroll
+        for (int s = 0; s < 3; ++s)
+            *reinterpret_cast<uint4*>(xs + (size_t)(s * m + r) * K + k) = make_uint4(t[s][0], t[s][1], t[s][2], t[s][3]);
+    }
+    __shared__ float part[4];
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0 && ssq) ssq[(size_t)blockIdx.x * m + r] = (part[0] + part[1]) + (part[2] + part[3]);
+}
+
+int split_rows(int m) { return npad_for(m); }
+int split_ssq_entries(int K) { return (K + 1023) / 1024; }
