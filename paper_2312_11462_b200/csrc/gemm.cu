@@ -334,12 +334,12 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     const bool dual = a.W2 != nullptr;
     if (dual != (a.epilogue == EPI_SWIGLU || a.epilogue == EPI_GEGLU)) return CSD_ERR_INVALID_ARG;
     if ((((uintptr_t)a.W) & 15) || (dual && (((uintptr_t)a.W2) & 15))) return CSD_ERR_INVALID_ARG;
-    if ((((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
     // kernel choice: the tensor-core kernel wherever it applies when selected (or, on automatic,
     // for blocks of more than AUTO_TC_MIN_ROWS rows, where the CUDA-core kernel is ALU-bound)
     const int path = gemm_path();
-    if (path != 1 && tc_supported(a.m, a.N, a.K, dual) && (path == 2 || a.m > AUTO_TC_MIN_ROWS))
+    if (path != 1 && a.xs && tc_supported(a.m, a.N, a.K, dual) && (path == 2 || a.m > AUTO_TC_MIN_ROWS))
         return launch_linear_tc(a, st);
+    if ((((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
     const LinearPlan pl = plan_linear(a.m, a.N, a.K, dual);
     if (pl.kslices > 1 && (!a.partial || !a.tickets)) return CSD_ERR_INVALID_ARG;
     GemmParams gp;
@@ -369,25 +369,39 @@ extern "C" csd_status csd_set_gemm_path(int path) {
     return CSD_OK;
 }
 
-extern "C" size_t csd_linear_workspace_bytes(int m, int N, int K) {
-    if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8) return 0;
-    return linear_scratch_bytes(m, N, K, false) + align_up((size_t)linear_ticket_count(N) * sizeof(unsigned), 256);
+struct LinearWs { size_t tickets, partial, xs, ssq, total; };
+static LinearWs linear_ws(int m, int N, int K) {
+    LinearWs w;
+    size_t off = 0;
+    w.tickets = off; off += align_up((size_t)linear_ticket_count(N) * sizeof(unsigned), 256);
+    w.partial = off; off += linear_scratch_bytes(m, N, K, false);
+    w.xs = off;      off += align_up((size_t)3 * CSD_MAX_ROWS * K * 2, 256);
+    w.ssq = off;     off += align_up((size_t)split_ssq_entries(K) * CSD_MAX_ROWS * sizeof(float), 256);
+    w.total = off;
+    return w;
 }
 
-// The ticket words at the start of the workspace must be zero before the first call; every
-// launch leaves them zero again, so one cudaMemset after allocation is enough.
+extern "C" size_t csd_linear_workspace_bytes(int m, int N, int K) {
+    if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8) return 0;
+    return linear_ws(m, N, K).total;
+}
+
+// The workspace must be zero before the first call (the ticket words live in it); every launch
+// leaves the tickets zero again, so one cudaMemset after allocation is enough.
 extern "C" csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, int m, float* Y_dev,
                                  void* workspace_dev, size_t workspace_bytes, void* stream) {
     if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8 || (K & 7)) return CSD_ERR_INVALID_ARG;
-    if (!W_bf16_dev || !X_dev || !Y_dev) return CSD_ERR_INVALID_ARG;
-    size_t need = csd_linear_workspace_bytes(m, N, K);
-    if (workspace_bytes < need || (need && !workspace_dev)) return CSD_ERR_CAPACITY;
+    if (!W_bf16_dev || !X_dev || !Y_dev || !workspace_dev) return CSD_ERR_INVALID_ARG;
+    const LinearWs w = linear_ws(m, N, K);
+    if (workspace_bytes < w.total) return CSD_ERR_CAPACITY;
     if (((uintptr_t)workspace_dev) & 255) return CSD_ERR_INVALID_ARG;
-    size_t toff = align_up((size_t)linear_ticket_count(N) * sizeof(unsigned), 256);
+    char* ws = (char*)workspace_dev;
     LinearArgs a;
     a.W = (const __nv_bfloat16*)W_bf16_dev; a.N = N; a.K = K; a.X = X_dev; a.ldx = K; a.m = m;
     a.Y = Y_dev; a.ldy = N; a.epilogue = EPI_STORE;
-    a.tickets = (unsigned*)workspace_dev;
-    a.partial = (float*)((char*)workspace_dev + toff);
+    a.tickets = (unsigned*)(ws + w.tickets);
+    a.partial = (float*)(ws + w.partial);
+    a.xs = (__nv_bfloat16*)(ws + w.xs);
+    a.ssq = (float*)(ws + w.ssq);
     return launch_linear(a, (cudaStream_t)stream);
 }

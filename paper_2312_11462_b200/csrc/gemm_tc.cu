@@ -506,3 +506,71 @@ split_rows_kernel(const float* __restrict__ X, int ldx, int K, int m, const __nv
 
 int split_rows(int m) { return npad_for(m); }
 int split_ssq_entries(int K) { return (K + 1023) / 1024; }
+
+static void pdl_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+}
+
+template <int M, bool DUAL>
+static csd_status launch_tc(const CUtensorMap& tw, const CUtensorMap& tw2, const CUtensorMap& tx, const TcParams& tp,
+                            const TcPlan& pl, cudaStream_t st) {
+    auto kern = skinny_gemm_tc_kernel<M, DUAL>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_MAX + 1024));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3((unsigned)pl.grid), dim3(TC_THREADS), pl.smem + 1024, st);
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, tw, tw2, tx, tp));
+    count_launch();
+    return CSD_OK;
+}
+
+csd_status launch_linear_tc(const LinearArgs& a, cudaStream_t st) {
+    const bool dual = a.W2 != nullptr;
+    if (!tc_supported(a.m, a.N, a.K, dual)) return CSD_ERR_UNSUPPORTED;
+    if (!a.xs || !a.partial || !a.tickets) return CSD_ERR_INVALID_ARG;
+    if ((((uintptr_t)a.xs) & 15)) return CSD_ERR_INVALID_ARG;
+    const TcPlan pl = tc_plan(a.m, a.N, a.K, dual);
+    CUtensorMap tw, tw2, tx;
+    if (!tensor_map_2d(a.W, a.N, a.K, TILE_N, &tw)) return CSD_ERR_UNSUPPORTED;
+    tw2 = tw;
+    if (dual && !tensor_map_2d(a.W2, a.N, a.K, TILE_N, &tw2)) return CSD_ERR_UNSUPPORTED;
+    if (!tensor_map_2d(a.xs, 3 * a.m, a.K, pl.npad, &tx)) return CSD_ERR_UNSUPPORTED;
+    int ssq_cnt = a.ssq_cnt;
+    if (!a.xs_ready) {
+        if (!a.X || (((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
+        if (a.gain && !a.ssq) return CSD_ERR_INVALID_ARG;
+        cudaLaunchConfig_t cfg;
+        cudaLaunchAttribute attr[1];
+        pdl_config(cfg, attr, dim3((unsigned)split_ssq_entries(a.K), (unsigned)a.m), dim3(128), 0, st);
+        CSD_CUDA(cudaLaunchKernelEx(&cfg, split_rows_kernel, a.X, a.ldx, a.K, a.m, a.gain, a.xs,
+                                    a.gain ? a.ssq : (float*)nullptr));
+        count_launch();
+        ssq_cnt = split_ssq_entries(a.K);
+    }
+    TcParams tp;
+    tp.Y = a.Y; tp.partial = a.partial; tp.tickets = a.tickets; tp.status = status_word_device();
+    tp.ssq_in = a.gain ? a.ssq : nullptr; tp.ssq_cnt = ssq_cnt;
+    tp.out_xs = a.out_xs; tp.out_gain = a.out_gain; tp.out_ssq = a.out_ssq; tp.out_ld = a.out_ld;
+    tp.N = a.N; tp.K = a.K; tp.ldy = a.ldy; tp.nkb = pl.kblocks; tp.tiles = pl.tiles; tp.stages = pl.stages;
+    tp.epilogue = a.epilogue; tp.eps = a.eps;
+#define CSD_TC_CASE(MM) \
+    case MM: return dual ? launch_tc<MM, true>(tw, tw2, tx, tp, pl, st) : launch_tc<MM, false>(tw, tw2, tx, tp, pl, st);
+    switch (a.m) {
+        CSD_TC_CASE(1) CSD_TC_CASE(2) CSD_TC_CASE(3) CSD_TC_CASE(4) CSD_TC_CASE(5) CSD_TC_CASE(6) CSD_TC_CASE(7)
+        CSD_TC_CASE(8) CSD_TC_CASE(9) CSD_TC_CASE(10) CSD_TC_CASE(11) CSD_TC_CASE(12) CSD_TC_CASE(13)
+        CSD_TC_CASE(14) CSD_TC_CASE(15) CSD_TC_CASE(16) CSD_TC_CASE(17)
+    }
+#undef CSD_TC_CASE
+    return CSD_ERR_INVALID_ARG;
+}
+
+}  // namespace csd
