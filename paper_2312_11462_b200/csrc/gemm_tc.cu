@@ -30,7 +30,7 @@ constexpr int TILE_N = 128;       // weight rows per MMA (its M dimension)
 constexpr int KB = 64;            // K elements per stage (one 128-byte swizzle atom wide)
 constexpr int STAGE_BYTES = TILE_N * KB * 2;      // 16 KB
 constexpr int SPIN_LIMIT = 20000000;              // bounded waits (about a second)
-constexpr size_t TC_SMEM_MAX = 224 * 1024;
+constexpr size_t TC_SMEM_MAX = 111 * 1024;              // two CTAs (of consecutive kernels) fit one SM
 
 static int g_path = 0;
 void set_gemm_path(int path) { g_path = path; }
@@ -61,7 +61,10 @@ static TcPlan tc_plan(int m, int N, int K, bool dual) {
     p.tiles = (N + TILE_N - 1) / TILE_N;
     p.kblocks = (K + KB - 1) / KB;
     const long long units = (long long)p.tiles * p.kblocks;
-    p.grid = (int)(units < tc_sm_count() ? units : tc_sm_count());
+    long long grid = units / 4;                           // at least four units per CTA
+    if (grid < 1) grid = 1;
+    if (grid > tc_sm_count()) grid = tc_sm_count();
+    p.grid = (int)grid;
     const size_t stage = (size_t)STAGE_BYTES * (dual ? 2 : 1) + (size_t)p.npad * 128;
     p.stages = (int)((TC_SMEM_MAX - 1024) / stage);
     if (p.stages > 12) p.stages = 12;
@@ -72,7 +75,9 @@ static TcPlan tc_plan(int m, int N, int K, bool dual) {
 
 bool tc_supported(int m, int N, int K, bool dual) {
     (void)dual;
-    return m >= 1 && m <= CSD_MAX_ROWS && N >= 1 && K >= 64 && (K & 7) == 0;
+    if (!(m >= 1 && m <= CSD_MAX_ROWS && N >= 1 && K >= 64 && (K & 7) == 0)) return false;
+    const long long units = (long long)((N + TILE_N - 1) / TILE_N) * ((K + KB - 1) / KB);
+    return units * (tc_sm_count() + 1) < (1LL << 31);
 }
 
 size_t tc_scratch_bytes(int m, int N, int K, bool dual) {
@@ -224,16 +229,17 @@ __device__ __forceinline__ void split3(float x, uint16_t& b1, uint16_t& b2, uint
 // Units of work are (tile of 128 output columns, 64-wide K block) pairs in tile-major order; CTA c
 // owns the contiguous range [unit_begin(c), unit_begin(c+1)), so every SM streams the same
 // number of weight bytes whatever N and K are.
-__device__ __forceinline__ long long unit_begin(int c, long long units, int ctas) { return (long long)c * units / ctas; }
-__device__ __forceinline__ int cta_of_unit(long long u, long long units, int ctas) {
-    int c = (int)(((u + 1) * ctas - 1) / units);
+// (units * ctas fits 32 bits: the planner refuses shapes where it would not)
+__device__ __forceinline__ unsigned unit_begin(unsigned c, unsigned units, unsigned ctas) { return c * units / ctas; }
+__device__ __forceinline__ int cta_of_unit(unsigned u, unsigned units, unsigned ctas) {
+    unsigned c = ((u + 1) * ctas - 1) / units;
     while (c + 1 < ctas && unit_begin(c + 1, units, ctas) <= u) ++c;
     while (c > 0 && unit_begin(c, units, ctas) > u) --c;
-    return c;
+    return (int)c;
 }
 
 template <int M, bool DUAL>
-__global__ void __launch_bounds__(TC_THREADS, 1)
+__global__ void __launch_bounds__(TC_THREADS, 2)
 skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmW2,
                       const __grid_constant__ CUtensorMap tmX, const TcParams p) {
     constexpr int NPAD = 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : (3 * M <= 48 ? 48 : 64));
@@ -251,8 +257,8 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, ctas = gridDim.x;
-    const long long units = (long long)p.tiles * p.nkb;
-    const long long u0 = unit_begin(cta, units, ctas), u1 = unit_begin(cta + 1, units, ctas);
+    const unsigned units = (unsigned)p.tiles * (unsigned)p.nkb;
+    const unsigned u0 = unit_begin(cta, units, ctas), u1 = unit_begin(cta + 1, units, ctas);
     const int items = (int)(u1 - u0);
 
     if (tid == 0) {
@@ -279,7 +285,7 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         if (lane == 0) {
             const int pre = items < p.stages ? items : p.stages;
             for (int i = 0; i < pre; ++i) {
-                const long long u = u0 + i;
+                const unsigned u = u0 + i;
                 const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
                 unsigned char* dst = ring + (size_t)i * STAGE;
                 mbar_expect_tx(&ctl->full[i], (uint32_t)STAGE);
@@ -292,7 +298,7 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             for (int i = pre; i < items && !*abort_flag; ++i) {
                 const int s = i % p.stages;
                 if (!mbar_wait(&ctl->empty[s], ((i / p.stages) - 1) & 1)) { *abort_flag = 1; break; }
-                const long long u = u0 + i;
+                const unsigned u = u0 + i;
                 const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
                 unsigned char* dst = ring + (size_t)s * STAGE;
                 mbar_expect_tx(&ctl->full[s], (uint32_t)STAGE);
@@ -386,29 +392,41 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     for (int r = 0; r < M; ++r) mine[(u * M + r) * TILE_N + col] = sums[u][r];
                 __threadfence();
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int c_lo = cta_of_unit((long long)tile * p.nkb, units, ctas);
-                const int c_hi = cta_of_unit((long long)(tile + 1) * p.nkb - 1, units, ctas);
+                const int c_lo = cta_of_unit((unsigned)tile * p.nkb, units, ctas);
+                const int c_hi = cta_of_unit((unsigned)(tile + 1) * p.nkb - 1, units, ctas);
                 if (et == 0) {
                     const unsigned old = atomicAdd(&p.tickets[tile], 1u);
                     ctl->last_flag = (old == (unsigned)(c_hi - c_lo));
                     if (ctl->last_flag) p.tickets[tile] = 0u;
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int last = ctl->last_flag;
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                const int last = ctl->last_flag;        // (rewritten only after every warp has passed the next bar.sync)
                 if (!last) continue;
                 __threadfence();
 #pragma unroll
                 for (int u = 0; u < NT; ++u)
 #pragma unroll
                     for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
-                for (int c = c_lo; c <= c_hi; ++c) {
-                    const int slot = (int)(unit_begin(c, units, ctas) / p.nkb) == tile ? 0 : 1;
-                    const float* src = p.partial + ((size_t)c * 2 + slot) * NT * M * TILE_N + col;
+                // parts in CTA order, a few contributors' loads in flight at a time
+                constexpr int CH = NT * M <= 12 ? 4 : (NT * M <= 24 ? 2 : 1);
+                for (int c = c_lo; c <= c_hi; c += CH) {
+                    float part[CH][NT * M];
 #pragma unroll
-                    for (int u = 0; u < NT; ++u)
+                    for (int h = 0; h < CH; ++h) {
+                        const int cc = min(c + h, c_hi);
+                        const int slot = (int)(unit_begin(cc, units, ctas) / p.nkb) == tile ? 0 : 1;
+                        const float* src = p.partial + ((size_t)cc * 2 + slot) * NT * M * TILE_N + col;
 #pragma unroll
-                        for (int r = 0; r < M; ++r) sums[u][r] += __ldcg(src + (u * M + r) * TILE_N);
+                        for (int v = 0; v < NT * M; ++v) part[h][v] = __ldcg(src + v * TILE_N);
+                    }
+#pragma unroll
+                    for (int h = 0; h < CH; ++h)
+                        if (c + h <= c_hi) {
+#pragma unroll
+                            for (int u = 0; u < NT; ++u)
+#pragma unroll
+                                for (int r = 0; r < M; ++r) sums[u][r] += part[h][u * M + r];
+                        }
                 }
             }
             // ---- finish the tile: this thread owns output column n for all M rows
