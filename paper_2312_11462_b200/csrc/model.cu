@@ -132,7 +132,7 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
-        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, total;
+        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, total;
     size_t layer_kv, layer_x;
 };
 
@@ -161,6 +161,9 @@ static WsLayout ws_layout(const csd_model_config& c) {
     size_t keys = c.max_seq > c.max_enc_len ? c.max_seq : c.max_enc_len;
     L.attn_partial = put(attn_scratch_bytes((int)keys, (int)H, (int)Dh));
     L.attn_tickets = put(H * 4);
+    const size_t kmax = d > di ? (d > ff ? d : ff) : (di > ff ? di : ff);
+    L.xs_tmp = put(3 * R * kmax * 2);
+    L.ssq_tmp = put((size_t)split_ssq_entries((int)kmax) * R * 4);
     if (c.arch == 0) {
         L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
         L.rope_s = put((size_t)c.max_seq * (Dh / 2) * 4);
@@ -203,6 +206,7 @@ static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat
     LinearArgs a;
     a.W = W; a.W2 = W2; a.N = N; a.K = K; a.X = X; a.ldx = ldx; a.m = m; a.gain = gain; a.eps = M->cfg.norm_eps;
     a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.partial = M->gemm_partial; a.tickets = M->gemm_tickets;
+    a.xs = M->xs_tmp; a.ssq = M->ssq_tmp;
     ProfScope ps(M, 0, st);
     if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
     return launch_linear(a, st);
@@ -292,6 +296,7 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     M->x = (float*)(ws + L.x); M->qkv = (float*)(ws + L.qkv); M->attn = (float*)(ws + L.attn);
     M->act = (float*)(ws + L.act);
     M->gemm_partial = (float*)(ws + L.gemm_partial); M->gemm_tickets = (unsigned*)(ws + L.gemm_tickets);
+    M->xs_tmp = (__nv_bfloat16*)(ws + L.xs_tmp); M->ssq_tmp = (float*)(ws + L.ssq_tmp);
     M->attn_partial = (float*)(ws + L.attn_partial); M->attn_tickets = (unsigned*)(ws + L.attn_tickets);
     M->status = status;
     cudaStream_t st = (cudaStream_t)stream;

@@ -27,6 +27,8 @@ struct csd_model {
     float *rope_c = nullptr, *rope_s = nullptr, *dec_bias = nullptr, *enc_bias = nullptr;
     float *gemm_partial = nullptr, *attn_partial = nullptr;
     unsigned *gemm_tickets = nullptr, *attn_tickets = nullptr;
+    __nv_bfloat16* xs_tmp = nullptr;    // three-term bf16 split of a GEMM's input rows (tensor-core path)
+    float* ssq_tmp = nullptr;           // pieces of the rows' sums of squares written with it
     int* status = nullptr;
     // optional per-kernel-class timing (csd_model_profile): event pairs around every launch
     bool prof = false;

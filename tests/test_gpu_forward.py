@@ -11,11 +11,14 @@ from gpu_util import LOGIT_MAX_ABS, LOGIT_REL_L2, rel_l2, require_gpu, to_dev_i3
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def b():
+@pytest.fixture(scope="module", params=[1, 2], ids=["cuda-core", "tensor-core"])
+def b(request):
+    """Every test here runs once per GEMM kernel: 128-bit loads + fp32 FMA, and TMA + tcgen05."""
     require_gpu()
     from paper_2312_11462_b200 import binding
-    return binding
+    binding.csd_set_gemm_path(request.param)
+    yield binding
+    binding.csd_set_gemm_path(0)
 
 
 def check(got, ref, what):

@@ -8,11 +8,14 @@ from gpu_util import rel_l2, require_gpu
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module")
-def b():
+@pytest.fixture(scope="module", params=[1, 2], ids=["cuda-core", "tensor-core"])
+def b(request):
+    """Every test here runs once per GEMM kernel: 128-bit loads + fp32 FMA, and TMA + tcgen05."""
     require_gpu()
     from paper_2312_11462_b200 import binding
-    return binding
+    binding.csd_set_gemm_path(request.param)
+    yield binding
+    binding.csd_set_gemm_path(0)
 
 
 def case(b, orc, m, N, K, seed):
@@ -26,7 +29,8 @@ def case(b, orc, m, N, K, seed):
     ref = orc.linear(orc.blob_to_u16(W).reshape(N, K), X.cpu().numpy())
     got = Y.cpu().numpy()
     # fp32 accumulation of K products of magnitude |w||x|: error ~ sqrt(K) * 2^-24 * |y|
-    assert rel_l2(got, ref) < 2e-6, (m, N, K)
+    # (the tensor cores add partial products with a little less care than an fp32 FMA chain)
+    assert rel_l2(got, ref) < 5e-6, (m, N, K)
     assert np.abs(got - ref).max() < 1e-4 * max(1.0, np.abs(ref).max())
 
 
