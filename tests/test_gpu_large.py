@@ -38,12 +38,37 @@ def test_7b_shaped_cascade_and_logits(b, orc):
     # teacher-forced: the target's logits over the oracle's own sequence, block by block
     seq = np.concatenate([prompt, want]).astype(np.int32)
     gm, om = gms[0], orc.Model(ts, orc.blob_to_u16(tb))
+    # Two implementations that each round K/V to bf16 cannot stay closer than a few 1e-3 in a deep
+    # stack: a relative difference delta upstream flips a fraction ~delta * 2^8 of the cache roundings,
+    # each flip is worth 2^-8, so the cache differs by ~sqrt(delta) * 2^-4 in rms, which feeds the next
+    # layer; the fixed point of that loop is (2^-4 * s)^2 with s <= 1 the attention's share of the
+    # signal, i.e. 1e-3 .. 4e-3.  Hence 5e-3 here, and the 2e-3 bound on the shallow stack below.
     for pos, m in ((0, 11), (11, 5), (16, 2)):
         blk = seq[pos:pos + m]
         g = gm.csd_review_forward(to_dev_i32(blk), pos).cpu().numpy()
         r = om.review_forward(blk, pos)
-        assert rel_l2(g, r) <= LOGIT_REL_L2, (pos, rel_l2(g, r))
+        assert rel_l2(g, r) <= 5e-3, (pos, rel_l2(g, r))
         assert np.abs(g - r).max() <= LOGIT_MAX_ABS
+
+
+@pytest.mark.parametrize("path", [1, 2], ids=["cuda-core", "tensor-core"])
+def test_7b_width_shallow_stack(b, orc, path):
+    # the 7B layer shapes (d 4096, 32 heads x 128, ffn 11008, vocabulary 32000) in a 3-layer stack
+    shape = llama_shape(3, 4096, 32, 11008, 32000, 64)
+    blob = workloads.make_weights(shape, seed=100, device="cuda")
+    seq = workloads.make_prompt(shape.vocab, 24, seed=1000)
+    b.csd_set_gemm_path(path)
+    try:
+        gm, om = b.Model(shape, blob), orc.Model(shape, orc.blob_to_u16(blob))
+        for pos, m in ((0, 17), (17, 5), (22, 1)):
+            blk = seq[pos:pos + m]
+            g = gm.csd_review_forward(to_dev_i32(blk), pos).cpu().numpy()
+            r = om.review_forward(blk, pos)
+            assert rel_l2(g, r) <= LOGIT_REL_L2, (pos, rel_l2(g, r))
+            assert np.abs(g - r).max() <= LOGIT_MAX_ABS
+        assert b.csd_device_status() == 0
+    finally:
+        b.csd_set_gemm_path(0)
 
 
 def test_long_cache_review_blocks(b, orc):
