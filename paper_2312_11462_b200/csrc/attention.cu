@@ -26,10 +26,22 @@ template <int DH> struct AttnCfg {
 
 struct AttnParams {
     const float* q; const __nv_bfloat16* Kc; const __nv_bfloat16* Vc; const float* bias; float* out;
+    __nv_bfloat16* out_xs; int out_xs_ld;
     float* partial; unsigned* tickets;
     int ldq, m, cap, H, n_keys, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
 };
+
+// two neighbouring output columns of row r as three bf16 terms each (rows term * m + r)
+__device__ __forceinline__ void store_split(__nv_bfloat16* xs, int ld, int m, int r, int col, float a, float b) {
+    uint16_t a1, a2, a3, c1, c2, c3;
+    split3(a, a1, a2, a3);
+    split3(b, c1, c2, c3);
+    uint32_t* base = reinterpret_cast<uint32_t*>(reinterpret_cast<uint16_t*>(xs) + col);
+    base[((size_t)r * ld) >> 1] = a1 | ((uint32_t)c1 << 16);
+    base[((size_t)(m + r) * ld) >> 1] = a2 | ((uint32_t)c2 << 16);
+    base[((size_t)(2 * m + r) * ld) >> 1] = a3 | ((uint32_t)c3 << 16);
+}
 
 template <int DH>
 __global__ void __launch_bounds__(AT)
@@ -173,6 +185,7 @@ block_attention_kernel(const AttnParams p) {
                 const float inv = row_l[r] > 0.f ? 1.f / row_l[r] : 0.f;
                 float* o = p.out + (size_t)r * p.ldo + h * DH + 2 * dp;
                 o[0] = acc[rr][0] * inv; o[1] = acc[rr][1] * inv;
+                if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, m, r, h * DH + 2 * dp, o[0], o[1]);
             }
         }
         return;
@@ -214,7 +227,16 @@ block_attention_kernel(const AttnParams p) {
                 den = fmaf(__ldcg(rec + DH + 1), w, den);
             }
         }
-        p.out[(size_t)r * p.ldo + h * DH + d] = den > 0.f ? num / den : 0.f;
+        const float o = den > 0.f ? num / den : 0.f;
+        p.out[(size_t)r * p.ldo + h * DH + d] = o;
+        if (p.out_xs) {
+            uint16_t b1, b2, b3;
+            split3(o, b1, b2, b3);
+            uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
+            xs[(size_t)r * p.out_xs_ld] = b1;
+            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
+            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
+        }
     }
 }
 
@@ -256,7 +278,7 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     ap.q = a.q; ap.Kc = a.Kc; ap.Vc = a.Vc; ap.bias = a.bias; ap.out = a.out; ap.partial = a.partial;
     ap.tickets = a.tickets; ap.ldq = a.ldq; ap.m = a.m; ap.cap = a.cap; ap.H = a.H; ap.n_keys = a.n_keys;
     ap.causal = a.causal; ap.bias_len = a.bias_len; ap.bias_zero = a.bias_zero; ap.q_pos0 = a.q_pos0;
-    ap.ldo = a.ldo; ap.scale = a.scale;
+    ap.ldo = a.ldo; ap.scale = a.scale; ap.out_xs = a.out_xs; ap.out_xs_ld = a.out_xs_ld;
     ap.nsplit = attn_splits(total, a.H);
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;

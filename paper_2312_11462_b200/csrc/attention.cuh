@@ -18,6 +18,8 @@ struct AttnArgs {
     int q_pos0 = 0;                       // position of row 0 (for the bias)
     float* out = nullptr;                 // [m, ldo]
     int ldo = 0;
+    __nv_bfloat16* out_xs = nullptr;      // optional: the output rows as three bf16 terms, row = term * m + r
+    int out_xs_ld = 0;
     float* partial = nullptr;             // split scratch (attn_scratch_bytes)
     unsigned* tickets = nullptr;          // H zero-initialised words
     int max_keys = 0;                     // capacity used to size the scratch

@@ -53,6 +53,15 @@ __device__ __forceinline__ uint16_t float_to_bf16_bits(float f) {
     return __bfloat16_as_ushort(__float2bfloat16_rn(f));
 }
 
+// x = b1 + b2 + b3 with bf16 terms (8 + 8 + 8 mantissa bits: exact for an fp32 value); the
+// tensor-core GEMM takes its fp32 rows in this form
+__device__ __forceinline__ void split3(float x, uint16_t& b1, uint16_t& b2, uint16_t& b3) {
+    b1 = float_to_bf16_bits(x);
+    const float r1 = x - bf16_bits_to_float(b1);
+    b2 = float_to_bf16_bits(r1);
+    b3 = float_to_bf16_bits(r1 - bf16_bits_to_float(b2));
+}
+
 // 128-bit streaming load that does not allocate in L1 (weights are read exactly once)
 __device__ __forceinline__ uint4 ldg_stream(const void* p) {
     uint4 v;

@@ -328,6 +328,11 @@ size_t linear_scratch_bytes(int m, int N, int K, bool dual) {
 
 int linear_ticket_count(int N) { return N + 1; }   // one ticket per row group, at least one row each
 
+bool linear_uses_tensor_cores(int m, int N, int K, bool dual) {
+    const int path = gemm_path();
+    return path != 1 && tc_supported(m, N, K, dual) && (path == 2 || m > AUTO_TC_MIN_ROWS);
+}
+
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     if (!a.W || !a.X || !a.Y || a.m < 1 || a.m > CSD_MAX_ROWS || a.N < 1 || a.K < 8 || (a.K & 7))
         return CSD_ERR_INVALID_ARG;
@@ -336,9 +341,7 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     if ((((uintptr_t)a.W) & 15) || (dual && (((uintptr_t)a.W2) & 15))) return CSD_ERR_INVALID_ARG;
     // kernel choice: the tensor-core kernel wherever it applies when selected (or, on automatic,
     // for blocks of more than AUTO_TC_MIN_ROWS rows, where the CUDA-core kernel is ALU-bound)
-    const int path = gemm_path();
-    if (path != 1 && a.xs && tc_supported(a.m, a.N, a.K, dual) && (path == 2 || a.m > AUTO_TC_MIN_ROWS))
-        return launch_linear_tc(a, st);
+    if (a.xs && linear_uses_tensor_cores(a.m, a.N, a.K, dual)) return launch_linear_tc(a, st);
     if ((((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
     const LinearPlan pl = plan_linear(a.m, a.N, a.K, dual);
     if (pl.kslices > 1 && (!a.partial || !a.tickets)) return CSD_ERR_INVALID_ARG;

@@ -37,5 +37,6 @@ int split_ssq_entries(int K);            // ssq pieces the stand-alone split ker
 size_t linear_scratch_bytes(int m, int N, int K, bool dual);
 int linear_ticket_count(int N);
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st);
+bool linear_uses_tensor_cores(int m, int N, int K, bool dual);   // the kernel launch_linear would pick (given a.xs)
 
 }  // namespace csd

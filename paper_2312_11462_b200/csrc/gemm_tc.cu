@@ -218,14 +218,6 @@ __device__ __forceinline__ float tc_gelu(float x) {
 }
 __device__ __forceinline__ float tc_silu(float x) { return x / (1.f + expf(-x)); }
 
-// x = b1 + b2 + b3 with bf16 terms (8 + 8 + 8 mantissa bits: exact for an fp32 value)
-__device__ __forceinline__ void split3(float x, uint16_t& b1, uint16_t& b2, uint16_t& b3) {
-    b1 = float_to_bf16_bits(x);
-    const float r1 = x - bf16_bits_to_float(b1);
-    b2 = float_to_bf16_bits(r1);
-    b3 = float_to_bf16_bits(r1 - bf16_bits_to_float(b2));
-}
-
 // Units of work are (tile of 128 output columns, 64-wide K block) pairs in tile-major order; CTA c
 // owns the contiguous range [unit_begin(c), unit_begin(c+1)), so every SM streams the same
 // number of weight bytes whatever N and K are.
