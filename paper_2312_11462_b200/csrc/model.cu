@@ -132,7 +132,7 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
-        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, total;
+        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, total;
     size_t layer_kv, layer_x;
 };
 
@@ -164,6 +164,10 @@ static WsLayout ws_layout(const csd_model_config& c) {
     const size_t kmax = d > di ? (d > ff ? d : ff) : (di > ff ? di : ff);
     L.xs_tmp = put(3 * R * kmax * 2);
     L.ssq_tmp = put((size_t)split_ssq_entries((int)kmax) * R * 4);
+    L.xs_x = put(3 * R * d * 2);
+    L.xs_attn = put(3 * R * di * 2);
+    L.xs_act = put(3 * R * ff * 2);
+    L.ssq_x = put(4 * ((d + 127) / 128) * R * 4);
     if (c.arch == 0) {
         L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
         L.rope_s = put((size_t)c.max_seq * (Dh / 2) * 4);
@@ -200,13 +204,30 @@ static csd_status check_config(const csd_model_config* c) {
     return CSD_OK;
 }
 
+// Hand-over of activations between kernels on the tensor-core path: a GEMM may receive its rows
+// already split into three bf16 terms (by the kernel that produced them) and may emit its own
+// result in that form, times the gain of the norm that follows, with the pieces of the rows' sums
+// of squares that norm needs.
+struct LinOpt {
+    const __nv_bfloat16* xs_in = nullptr; const float* ssq_in = nullptr; int ssq_cnt = 0;
+    __nv_bfloat16* out_xs = nullptr; int out_ld = 0; const __nv_bfloat16* out_gain = nullptr; float* out_ssq = nullptr;
+};
+
 // One linear layer of the forward; all of them share the model's split scratch.
 static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat16* W2, int N, int K, const float* X,
-                         int ldx, int m, const __nv_bfloat16* gain, float* Y, int ldy, int epi, cudaStream_t st) {
+                         int ldx, int m, const __nv_bfloat16* gain, float* Y, int ldy, int epi, cudaStream_t st,
+                         const LinOpt* o = nullptr) {
     LinearArgs a;
     a.W = W; a.W2 = W2; a.N = N; a.K = K; a.X = X; a.ldx = ldx; a.m = m; a.gain = gain; a.eps = M->cfg.norm_eps;
     a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.partial = M->gemm_partial; a.tickets = M->gemm_tickets;
     a.xs = M->xs_tmp; a.ssq = M->ssq_tmp;
+    if (o) {
+        if (o->xs_in) {
+            a.xs = const_cast<__nv_bfloat16*>(o->xs_in); a.xs_ready = true;
+            a.ssq = const_cast<float*>(o->ssq_in); a.ssq_cnt = o->ssq_cnt;
+        }
+        a.out_xs = o->out_xs; a.out_ld = o->out_ld; a.out_gain = o->out_gain; a.out_ssq = o->out_ssq;
+    }
     ProfScope ps(M, 0, st);
     if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
     return launch_linear(a, st);
@@ -225,19 +246,37 @@ static csd_status attention(csd_model* M, const AttnArgs& a, cudaStream_t st) {
 
 // q|k|v projections of `m` rows with the norm fused; one GEMM when the three matrices are
 // contiguous in the blob (they are whenever d_inner * d_model is a multiple of 128).
-static csd_status project_qkv(csd_model* M, const LayerW& y, const float* X, int m, float* out, cudaStream_t st) {
+static csd_status project_qkv(csd_model* M, const LayerW& y, const float* X, int m, float* out, cudaStream_t st,
+                              const LinOpt* o = nullptr) {
     const int d = M->cfg.d_model, di = M->di;
     if (y.wk == y.wq + (size_t)di * d && y.wv == y.wk + (size_t)di * d)
-        return linear(M, y.wq, nullptr, 3 * di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st);
-    CSD_TRY(linear(M, y.wq, nullptr, di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st));
-    CSD_TRY(linear(M, y.wk, nullptr, di, d, X, d, m, y.norm1, out + di, 3 * di, EPI_STORE, st));
-    return linear(M, y.wv, nullptr, di, d, X, d, m, y.norm1, out + 2 * di, 3 * di, EPI_STORE, st);
+        return linear(M, y.wq, nullptr, 3 * di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st, o);
+    CSD_TRY(linear(M, y.wq, nullptr, di, d, X, d, m, y.norm1, out, 3 * di, EPI_STORE, st, o));
+    CSD_TRY(linear(M, y.wk, nullptr, di, d, X, d, m, y.norm1, out + di, 3 * di, EPI_STORE, st, o));
+    return linear(M, y.wv, nullptr, di, d, X, d, m, y.norm1, out + 2 * di, 3 * di, EPI_STORE, st, o);
 }
 
-static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, cudaStream_t st) {
+// Gated feed-forward with its norm, then the down projection added into the residual rows.
+// x_in: the rows already in three-term form (or null); next_gain: gain of the norm that reads the
+// residual rows next (the result is handed on in three-term form when the kernels allow it).
+// Returns through *x_out whether M->xs_x / M->ssq_x now describe the updated rows.
+static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, cudaStream_t st,
+                               bool x_in = false, const __nv_bfloat16* next_gain = nullptr, int next_N = 0,
+                               bool next_dual = false, bool* x_out = nullptr) {
     const int d = M->cfg.d_model, ff = M->cfg.d_ff;
-    CSD_TRY(linear(M, y.wgate, y.wup, ff, d, X, d, m, y.norm2, M->act, ff, M->cfg.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, st));
-    return linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, X, d, EPI_ADD, st);
+    const int cnt_d = 4 * ((d + 127) / 128);
+    const bool tc_up = linear_uses_tensor_cores(m, ff, d, true), tc_down = linear_uses_tensor_cores(m, d, ff, false);
+    LinOpt up;
+    if (x_in) { up.xs_in = M->xs_x; up.ssq_in = M->ssq_x; up.ssq_cnt = cnt_d; }
+    const bool act_ready = tc_up && tc_down;
+    if (act_ready) { up.out_xs = M->xs_act; up.out_ld = ff; }
+    CSD_TRY(linear(M, y.wgate, y.wup, ff, d, X, d, m, y.norm2, M->act, ff, M->cfg.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, st, &up));
+    LinOpt down;
+    if (act_ready) down.xs_in = M->xs_act;
+    const bool hand_on = tc_down && next_gain && linear_uses_tensor_cores(m, next_N, d, next_dual);
+    if (hand_on) { down.out_xs = M->xs_x; down.out_ld = d; down.out_gain = next_gain; down.out_ssq = M->ssq_x; }
+    if (x_out) *x_out = hand_on;
+    return linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, X, d, EPI_ADD, st, &down);
 }
 
 }  // namespace csd
@@ -297,6 +336,8 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     M->act = (float*)(ws + L.act);
     M->gemm_partial = (float*)(ws + L.gemm_partial); M->gemm_tickets = (unsigned*)(ws + L.gemm_tickets);
     M->xs_tmp = (__nv_bfloat16*)(ws + L.xs_tmp); M->ssq_tmp = (float*)(ws + L.ssq_tmp);
+    M->xs_x = (__nv_bfloat16*)(ws + L.xs_x); M->xs_attn = (__nv_bfloat16*)(ws + L.xs_attn);
+    M->xs_act = (__nv_bfloat16*)(ws + L.xs_act); M->ssq_x = (float*)(ws + L.ssq_x);
     M->attn_partial = (float*)(ws + L.attn_partial); M->attn_tickets = (unsigned*)(ws + L.attn_tickets);
     M->status = status;
     cudaStream_t st = (cudaStream_t)stream;
