@@ -476,11 +476,18 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
         count_launch();
     }
+    // x_ready: M->xs_x / M->ssq_x hold the residual rows (times the gain of the norm that reads them
+    // next) in three-term form, written by the epilogue of the GEMM that produced the rows
+    bool x_ready = false;
+    const int ff = c.d_ff, cnt_d = 4 * ((d + 127) / 128);
+    const bool tc_o = linear_uses_tensor_cores(m, d, di, false);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& y = M->dec[l];
         __nv_bfloat16* Kl = M->kcache + (size_t)l * M->layer_kv;
         __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
-        CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st));
+        LinOpt qo;
+        if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = cnt_d; }
+        CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         {
             ProfScope ps(M, 2, st);
             rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
@@ -493,21 +500,43 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         a.n_keys = kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
         if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = kv_len; }
         a.out = M->attn; a.ldo = di; a.partial = M->attn_partial; a.tickets = M->attn_tickets;
+        if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
         CSD_TRY(attention(M, a, st));
-        CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
+        // output projection into the residual rows; hands them on to the norm that follows
+        LinOpt oo;
+        if (tc_o) oo.xs_in = M->xs_attn;
+        const __nv_bfloat16* after_o = c.arch == 1 ? y.norm_x : y.norm2;
+        x_ready = tc_o && (c.arch == 1 ? linear_uses_tensor_cores(m, di, d, false) : linear_uses_tensor_cores(m, ff, d, true));
+        if (x_ready) { oo.out_xs = M->xs_x; oo.out_ld = d; oo.out_gain = after_o; oo.out_ssq = M->ssq_x; }
+        CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st, &oo));
         if (c.arch == 1) {
-            CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st));
+            LinOpt xq;
+            if (x_ready) { xq.xs_in = M->xs_x; xq.ssq_in = M->ssq_x; xq.ssq_cnt = cnt_d; }
+            CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st, &xq));
             AttnArgs x;
             x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
             x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
             x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di; x.partial = M->attn_partial;
             x.tickets = M->attn_tickets;
+            if (tc_o) { x.out_xs = M->xs_attn; x.out_xs_ld = di; }
             CSD_TRY(attention(M, x, st));
-            CSD_TRY(linear(M, y.xo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st));
+            LinOpt xo;
+            if (tc_o) xo.xs_in = M->xs_attn;
+            x_ready = tc_o && linear_uses_tensor_cores(m, ff, d, true);
+            if (x_ready) { xo.out_xs = M->xs_x; xo.out_ld = d; xo.out_gain = y.norm2; xo.out_ssq = M->ssq_x; }
+            CSD_TRY(linear(M, y.xo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st, &xo));
         }
-        CSD_TRY(feed_forward(M, y, M->x, m, st));
+        // feed-forward; its down projection hands the rows on to the next layer's first norm (or the final one)
+        const bool last = l + 1 == c.n_layers;
+        const __nv_bfloat16* next_gain = last ? M->final_norm : M->dec[l + 1].norm1;
+        const LayerW* nx = last ? nullptr : &M->dec[l + 1];
+        const bool fused_qkv = nx && nx->wk == nx->wq + (size_t)di * d && nx->wv == nx->wk + (size_t)di * d;
+        const int next_N = last ? V : (fused_qkv ? 3 * di : di);
+        CSD_TRY(feed_forward(M, y, M->x, m, st, x_ready, next_gain, next_N, false, &x_ready));
     }
-    CSD_TRY(linear(M, M->lm_head, nullptr, V, d, M->x, d, m, M->final_norm, logits_out_dev, V, EPI_STORE, st));
+    LinOpt ho;
+    if (x_ready) { ho.xs_in = M->xs_x; ho.ssq_in = M->ssq_x; ho.ssq_cnt = cnt_d; }
+    CSD_TRY(linear(M, M->lm_head, nullptr, V, d, M->x, d, m, M->final_norm, logits_out_dev, V, EPI_STORE, st, &ho));
     CSD_CUDA(cudaGetLastError());
     return CSD_OK;
 }
