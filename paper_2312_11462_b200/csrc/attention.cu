@@ -240,9 +240,11 @@ block_attention_kernel(const AttnParams p) {
     }
 }
 
+// One 64-key tile per CTA while that still gives no more than about two CTAs per SM: short caches
+// are latency-bound, and a CTA that walks several tiles pays one round trip per tile.
 int attn_splits(int total_keys, int H) {
     int by_sm = (2 * 148 + H - 1) / H;
-    int by_len = (total_keys + 127) / 128;
+    int by_len = (total_keys + TILE - 1) / TILE;
     int n = by_sm < by_len ? by_sm : by_len;
     if (n < 1) n = 1;
     if (n > MAX_SPLITS) n = MAX_SPLITS;
