@@ -64,6 +64,8 @@ block_attention_kernel(const AttnParams p) {
     const int s_begin = split * p.split_len;
     const int s_end = min(total, s_begin + p.split_len);
 
+    pdl_wait();       // q and the appended K/V rows come from the kernels before this one
+    pdl_trigger();
     for (int i = tid; i < m * DH; i += AT) qs[i] = p.q[(size_t)(i / DH) * p.ldq + h * DH + (i % DH)];
     if (tid < 32) { row_m[tid] = -INFINITY; row_l[tid] = 0.f; row_a[tid] = 1.f; }
 
@@ -264,10 +266,9 @@ static csd_status launch_dh(const AttnParams& ap, cudaStream_t st) {
         CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnCfg<DH>::SMEM));
         attr_set = true;
     }
-    dim3 grid((unsigned)ap.H, (unsigned)ap.nsplit);
-    kern<<<grid, AT, AttnCfg<DH>::SMEM, st>>>(ap);
+    PdlLaunch L(dim3((unsigned)ap.H, (unsigned)ap.nsplit), dim3(AT), AttnCfg<DH>::SMEM, st);
+    CSD_CUDA(cudaLaunchKernelEx(&L.cfg, kern, ap));
     count_launch();
-    CSD_CUDA(cudaGetLastError());
     return CSD_OK;
 }
 

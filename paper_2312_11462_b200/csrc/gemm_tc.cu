@@ -269,6 +269,10 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort_flag = &ctl->abort_flag;
+    // Let the next kernel in the stream start now: its CTAs take the second slot of each SM, set
+    // themselves up and request their first weight tiles while this kernel is still streaming;
+    // they touch nothing this kernel writes before their own dependency wait.
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     if (warp == 0) {
         // ---- TMA producer.  The weights do not depend on the kernel that produces the rows, so
@@ -461,7 +465,6 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             }
         }
     }
-    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     if (*abort_flag) {
         if (tid == 0) set_status(p.status, CSD_ERR_TIMEOUT);
         __nanosleep(2000000);          // let copies already in flight land before the CTA's memory is released

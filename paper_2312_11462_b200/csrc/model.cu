@@ -14,6 +14,8 @@ namespace csd {
 // ---------------------------------------------------------------------------------------------
 __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E, int V, int d,
                              float* __restrict__ x, int* status) {
+    pdl_wait();
+    pdl_trigger();
     const int r = blockIdx.x;
     int t = tokens[r];
     if (t < 0 || t >= V) {
@@ -48,6 +50,8 @@ __global__ void bias_table_kernel(const __nv_bfloat16* __restrict__ rel_bias, co
 __global__ void rope_append_kernel(float* __restrict__ src, int ld, int q_off, int k_off, int v_off, int Dh,
                                    int pos0, int cap, const float* __restrict__ cs, const float* __restrict__ sn,
                                    __nv_bfloat16* __restrict__ Kc, __nv_bfloat16* __restrict__ Vc) {
+    pdl_wait();
+    pdl_trigger();
     const int r = blockIdx.x, h = blockIdx.y, pos = pos0 + r, half = Dh / 2;
     float* row = src + (size_t)r * ld;
     __nv_bfloat16* kdst = Kc + ((size_t)h * cap + pos) * Dh;
@@ -490,9 +494,10 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         {
             ProfScope ps(M, 2, st);
-            rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
-                                                          c.arch == 0 ? M->rope_c : nullptr,
-                                                          c.arch == 0 ? M->rope_s : nullptr, Kl, Vl);
+            PdlLaunch L(dim3(m, H), dim3(64), 0, st);
+            CSD_CUDA(cudaLaunchKernelEx(&L.cfg, rope_append_kernel, M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
+                                        (const float*)(c.arch == 0 ? M->rope_c : nullptr),
+                                        (const float*)(c.arch == 0 ? M->rope_s : nullptr), Kl, Vl));
             count_launch();
         }
         AttnArgs a;
