@@ -536,6 +536,8 @@ static csd_status launch_tc(const CUtensorMap& tw, const CUtensorMap& tw2, const
     static bool attr_set = false;
     if (!attr_set) {
         CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)TC_SMEM_MAX + 1024));
+        // ask for the largest shared-memory carve-out, or the second CTA (the next kernel's) does not fit
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
         attr_set = true;
     }
     cudaLaunchConfig_t cfg;
