@@ -77,3 +77,135 @@ __device__ __forceinline__ UnitPos unit_pos(const ChainOpDev& o, unsigned u) {
     p.which = o.dual ? rem & 1 : 0;
     return p;
 }
+
+template <int M>
+__global__ void __launch_bounds__(TC_THREADS, 1)
+gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
+    constexpr int NPAD = 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : (3 * M <= 48 ? 48 : 64));
+    constexpr int ACC_COLS = 2 * NPAD;                         // room for the two matrices of a gated GEMM
+    constexpr int TMEM_COLS = 2 * ACC_COLS <= 64 ? 64 : (2 * ACC_COLS <= 128 ? 128 : 256);
+    constexpr int XBYTES = NPAD * 128;
+    constexpr int STAGE = STAGE_BYTES + XBYTES;
+    constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NPAD >> 3) << 17) |
+                               ((uint32_t)(TILE_N >> 4) << 24);
+
+    extern __shared__ unsigned char smem_raw[];
+    unsigned char* ring = (unsigned char*)(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+    ChainCtrl* ctl = (ChainCtrl*)(ring + (size_t)cp.stages * STAGE);
+
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const unsigned cta = blockIdx.x, ctas = gridDim.x;
+
+    if (tid == 0) {
+        for (int s = 0; s < 12; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
+        for (int b = 0; b < 2; ++b) { mbar_init(&ctl->acc_full[b], 1); mbar_init(&ctl->acc_empty[b], 4); }
+        ctl->abort_flag = 0; ctl->last_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&ctl->tmem_base)), "r"((uint32_t)TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = ctl->tmem_base;
+    volatile int* abort_flag = &ctl->abort_flag;
+
+    // this CTA's share of every GEMM of the chain
+    unsigned u0[CHAIN_MAX_OPS], cnt[CHAIN_MAX_OPS], units[CHAIN_MAX_OPS];
+    int total = 0;
+#pragma unroll
+    for (int j = 0; j < CHAIN_MAX_OPS; ++j) {
+        u0[j] = cnt[j] = units[j] = 0;
+        if (j < cp.n_ops) {
+            units[j] = (unsigned)cp.op[j].tiles * (unsigned)cp.op[j].nkb * (cp.op[j].dual ? 2u : 1u);
+            u0[j] = ch_unit_begin(cta, units[j], ctas);
+            cnt[j] = ch_unit_begin(cta + 1, units[j], ctas) - u0[j];
+            total += (int)cnt[j];
+        }
+    }
+
+    if (warp == 0) {
+        // ---- TMA producer: two cursors over this CTA's items of all GEMMs.  Weight tiles run
+        //      ahead as far as the ring allows; the rows' terms of GEMM j follow once GEMM j-1
+        //      has been reported finished by every CTA.
+        if (lane == 0) {
+            int gw = 0, wop = 0; unsigned wi = 0;      // next weight tile: global index, GEMM, index inside it
+            int gx = 0, xop = 0; unsigned xi = 0;      // next rows tile
+            int dep_ok_upto = 0;                       // rows of GEMMs <= this index may be loaded
+            int idle = 0;
+            while (wop < cp.n_ops && cnt[wop] == 0) ++wop;
+            while (xop < cp.n_ops && cnt[xop] == 0) ++xop;
+            while (gx < total && !*abort_flag) {
+                bool progressed = false;
+                if (gw < total) {
+                    const int s = gw % cp.stages;
+                    if (gw < cp.stages || mbar_test(&ctl->empty[s], ((gw / cp.stages) - 1) & 1)) {
+                        const ChainOpDev& o = cp.op[wop];
+                        const UnitPos up = unit_pos(o, u0[wop] + wi);
+                        mbar_expect_tx(&ctl->full[s], (uint32_t)STAGE);
+                        tma_load_2d(ring + (size_t)s * STAGE, up.which ? &o.tmW2 : &o.tmW, &ctl->full[s], up.kb * KB,
+                                    up.tile * TILE_N);
+                        ++gw;
+                        if (++wi == cnt[wop]) { wi = 0; do { ++wop; } while (wop < cp.n_ops && cnt[wop] == 0); }
+                        progressed = true;
+                    }
+                }
+                if (gx < gw) {
+                    if (xop > dep_ok_upto) {
+                        // GEMM xop reads what GEMM xop-1 wrote: has every CTA finished xop-1 ?
+                        if ((int)(ld_acquire(cp.done + (xop - 1)) - cp.done_target) >= 0) dep_ok_upto = xop;
+                    }
+                    if (xop <= dep_ok_upto) {
+                        const ChainOpDev& o = cp.op[xop];
+                        const UnitPos up = unit_pos(o, u0[xop] + xi);
+                        const int s = gx % cp.stages;
+                        tma_load_2d(ring + (size_t)s * STAGE + STAGE_BYTES, &o.tmX, &ctl->full[s], up.kb * KB, 0);
+                        ++gx;
+                        if (++xi == cnt[xop]) { xi = 0; do { ++xop; } while (xop < cp.n_ops && cnt[xop] == 0); }
+                        progressed = true;
+                    }
+                }
+                if (progressed) idle = 0;
+                else if (++idle > DEP_POLL_LIMIT) { *abort_flag = 1; break; }
+            }
+        }
+    } else if (warp == 1) {
+        // ---- MMA issuer: one accumulator set per segment (the part of a tile inside this CTA's share)
+        if (lane == 0) {
+            int gi = 0, seg = 0;
+            for (int j = 0; j < cp.n_ops && !*abort_flag; ++j) {
+                const ChainOpDev& o = cp.op[j];
+                const int per_tile = o.nkb * (o.dual ? 2 : 1);
+                unsigned i = 0;
+                while (i < cnt[j] && !*abort_flag) {
+                    const int b = seg & 1;
+                    const int rem = (int)((u0[j] + i) % per_tile);
+                    const int seg_len = min(per_tile - rem, (int)(cnt[j] - i));
+                    if (!mbar_wait(&ctl->acc_empty[b], ((seg >> 1) & 1) ^ 1)) { *abort_flag = 1; break; }
+                    tc_fence_after();
+                    const uint32_t d0 = tmem + (uint32_t)(b * ACC_COLS);
+                    bool started[2] = {false, false};
+                    for (int t = 0; t < seg_len; ++t, ++i, ++gi) {
+                        const int s = gi % cp.stages;
+                        if (!mbar_wait(&ctl->full[s], (gi / cp.stages) & 1)) { *abort_flag = 1; break; }
+                        tc_fence_after();
+                        const int which = o.dual ? (rem + t) & 1 : 0;
+                        const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE);
+                        const uint32_t b_addr = a_addr + STAGE_BYTES;
+#pragma unroll
+                        for (int k = 0; k < KB / 16; ++k)
+                            tc_mma(d0 + which * NPAD, smem_desc_sw128(a_addr + k * 32), smem_desc_sw128(b_addr + k * 32),
+                                   IDESC, (started[which] || k != 0) ? 1u : 0u);
+                        started[which] = true;
+                        tc_commit(&ctl->empty[s]);
+                    }
+                    if (*abort_flag) break;
+                    tc_commit(&ctl->acc_full[b]);
+                    ++seg;
+                }
+            }
+        }
+    } else {
