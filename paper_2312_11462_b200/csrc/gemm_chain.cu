@@ -209,3 +209,166 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
             }
         }
     } else {
+        // ---- epilogue warps: quadrant q of tensor memory holds weight rows q*32 .. q*32+31 of the tile
+        const int q = warp & 3, et = (warp - 2) * 32 + lane;
+        float* my_part = cp.partial + (size_t)cta * 2 * 2 * M * TILE_N;
+        int seg = 0;
+        bool dead = false;
+        for (int j = 0; j < cp.n_ops && !dead; ++j) {
+            const ChainOpDev& o = cp.op[j];
+            const int NT = o.dual ? 2 : 1, per_tile = o.nkb * NT;
+            unsigned i = 0;
+            int op_seg = 0;
+            while (i < cnt[j]) {
+                const int b = seg & 1;
+                const int tile = (int)((u0[j] + i) / per_tile), rem = (int)((u0[j] + i) % per_tile);
+                const int seg_len = min(per_tile - rem, (int)(cnt[j] - i));
+                i += seg_len;
+                if (!mbar_wait(&ctl->acc_full[b], (seg >> 1) & 1)) { *abort_flag = 1; dead = true; break; }
+                tc_fence_after();
+                if (op_seg == 0) {      // the rows of this GEMM are final by now: their rms-norm factors
+                    if (o.ssq_in && et < M) {
+                        float sq = 0.f;
+                        for (int c = 0; c < o.ssq_cnt; ++c) sq += __ldcg(o.ssq_in + (size_t)c * M + et);
+                        ctl->scale[et] = 1.f / sqrtf(sq / (float)o.K + o.eps);
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                }
+                // which of the two matrices of a gated GEMM this segment touched at all
+                const bool has0 = !o.dual || seg_len > 1 || (rem & 1) == 0;
+                const bool has1 = o.dual && (seg_len > 1 || (rem & 1) == 1);
+                const uint32_t taddr = tmem + ((uint32_t)(q * 32) << 16) + (uint32_t)(b * ACC_COLS);
+                float sums[2][M];
+#pragma unroll
+                for (int u = 0; u < 2; ++u) {
+#pragma unroll
+                    for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
+                    if (u == 0 ? !has0 : !has1) continue;
+                    float third[M], second[M];
+#pragma unroll
+                    for (int r = 0; r < M; ++r) { second[r] = 0.f; third[r] = 0.f; }
+#pragma unroll
+                    for (int c0 = 0; c0 < NPAD; c0 += 16) {
+                        if (c0 >= 3 * M) break;
+                        float v[16];
+                        tc_ld16(taddr + (uint32_t)(u * NPAD + c0), v);
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int col = c0 + c;
+                            if (col < M) sums[u][col] = v[c];
+                            else if (col < 2 * M) second[col - M] = v[c];
+                            else if (col < 3 * M) third[col - 2 * M] = v[c];
+                        }
+                    }
+#pragma unroll
+                    for (int r = 0; r < M; ++r) sums[u][r] += second[r] + third[r];
+                }
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) mbar_arrive(&ctl->acc_empty[b]);
+                const int col = q * 32 + lane, n = tile * TILE_N + col;
+                if (seg_len < per_tile) {
+                    // part of a tile: park it (slot 0 = this CTA's first segment of the GEMM, 1 = a later
+                    // one); whoever arrives last adds all parts in CTA order and finishes the tile
+                    float* mine = my_part + (size_t)(op_seg == 0 ? 0 : 1) * 2 * M * TILE_N;
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+                        if (u < NT) {
+#pragma unroll
+                            for (int r = 0; r < M; ++r) mine[(u * M + r) * TILE_N + col] = sums[u][r];
+                        }
+                    __threadfence();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int c_lo = ch_cta_of_unit((unsigned)tile * per_tile, units[j], ctas);
+                    const int c_hi = ch_cta_of_unit((unsigned)(tile + 1) * per_tile - 1, units[j], ctas);
+                    if (et == 0) {
+                        const unsigned old = atomicAdd(&o.tickets[tile], 1u);
+                        ctl->last_flag = (old == (unsigned)(c_hi - c_lo));
+                        if (ctl->last_flag) o.tickets[tile] = 0u;
+                    }
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    const int last = ctl->last_flag;
+                    ++seg; ++op_seg;
+                    if (!last) continue;
+                    __threadfence();
+#pragma unroll
+                    for (int u = 0; u < 2; ++u)
+#pragma unroll
+                        for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
+                    for (int c = c_lo; c <= c_hi; ++c) {
+                        const int slot = (int)(ch_unit_begin(c, units[j], ctas) / per_tile) == tile ? 0 : 1;
+                        const float* src = cp.partial + ((size_t)c * 2 + slot) * 2 * M * TILE_N + col;
+                        float part[2][M];
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+                            if (u < NT) {
+#pragma unroll
+                                for (int r = 0; r < M; ++r) part[u][r] = __ldcg(src + (u * M + r) * TILE_N);
+                            }
+#pragma unroll
+                        for (int u = 0; u < 2; ++u)
+                            if (u < NT) {
+#pragma unroll
+                                for (int r = 0; r < M; ++r) sums[u][r] += part[u][r];
+                            }
+                    }
+                } else {
+                    ++seg; ++op_seg;
+                }
+                // ---- finish the tile: this thread owns output column n for all M rows
+                float outv[M];
+#pragma unroll
+                for (int r = 0; r < M; ++r) {
+                    const float scale = o.ssq_in ? ctl->scale[r] : 1.f;
+                    float val = sums[0][r] * scale;
+                    if (o.dual) {
+                        const float up = sums[1][r] * scale;
+                        val = (o.epilogue == EPI_GEGLU ? ch_gelu(val) : ch_silu(val)) * up;
+                    }
+                    if (n < o.N) {
+                        float* y = o.Y + (size_t)r * o.ldy + n;
+                        if (o.epilogue == EPI_ADD) val += *y;
+                        *y = val;
+                    } else {
+                        val = 0.f;
+                    }
+                    outv[r] = val;
+                }
+                if (o.out_ssq) {
+#pragma unroll
+                    for (int r = 0; r < M; ++r) {
+                        const float sq = warp_sum(outv[r] * outv[r]);
+                        if (lane == 0) o.out_ssq[(size_t)(tile * 4 + q) * M + r] = sq;
+                    }
+                }
+                if (o.out_xs && n < o.N) {
+                    const float g = o.out_gain ? __bfloat162float(o.out_gain[n]) : 1.f;
+#pragma unroll
+                    for (int r = 0; r < M; ++r) {
+                        uint16_t b1, b2, b3;
+                        split3(outv[r] * g, b1, b2, b3);
+                        uint16_t* dst = reinterpret_cast<uint16_t*>(o.out_xs) + n;
+                        dst[(size_t)r * o.out_ld] = b1;
+                        dst[(size_t)(M + r) * o.out_ld] = b2;
+                        dst[(size_t)(2 * M + r) * o.out_ld] = b3;
+                    }
+                }
+            }
+            if (dead) break;
+            // report this GEMM finished by this CTA (its own tiles and any fix-ups it performed)
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (et == 0) atomicAdd(cp.done + j, 1u);
+        }
+    }
+    if (*abort_flag) {
+        if (tid == 0) set_status(cp.status, CSD_ERR_TIMEOUT);
+        __nanosleep(2000000);
+    }
+    tc_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tc_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
+    }
+}
