@@ -13,6 +13,7 @@
 // stops, frees its tensor memory and returns.
 #include "gemm_tc.cuh"
 #include "tc_common.cuh"
+#include <string.h>
 
 namespace csd {
 
@@ -372,3 +373,88 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem), "r"((uint32_t)TMEM_COLS) : "memory");
     }
 }
+
+static int chain_npad(int m) { int c = 3 * m; return c <= 16 ? 16 : (c <= 32 ? 32 : (c <= 48 ? 48 : 64)); }
+
+size_t chain_scratch_bytes(int m) {
+    return align_up((size_t)tc_sm_count() * 2 * 2 * m * TILE_N * sizeof(float), 256);
+}
+
+template <int M>
+static csd_status launch_chain_m(const ChainParams& cp, int grid, size_t smem, cudaStream_t st) {
+    auto kern = gemm_chain_kernel<M>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)CHAIN_SMEM + 1024));
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributePreferredSharedMemoryCarveout, cudaSharedmemCarveoutMaxShared));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)grid);
+    cfg.blockDim = dim3(TC_THREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeCooperative;      // every CTA resident at once: they wait for one another
+    attr[0].val.cooperative = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, cp));
+    count_launch();
+    return CSD_OK;
+}
+
+// ops[j+1] must read (a.xs) what ops[j] writes (a.out_xs); ops[0].xs must be ready.  done_dev:
+// CHAIN_MAX_OPS zero-initialised counters owned by the caller, epoch_host: launches so far.
+csd_status launch_linear_chain(const LinearArgs* ops, int n_ops, unsigned* done_dev, unsigned* epoch_host,
+                               cudaStream_t st) {
+    if (!ops || n_ops < 1 || n_ops > CHAIN_MAX_OPS || !done_dev || !epoch_host) return CSD_ERR_INVALID_ARG;
+    const int m = ops[0].m, grid = tc_sm_count();
+    if (m < 1 || m > CSD_MAX_ROWS) return CSD_ERR_INVALID_ARG;
+    const int npad = chain_npad(m);
+    ChainParams cp;
+    memset(&cp, 0, sizeof(cp));
+    size_t ticket_off = 0;
+    for (int j = 0; j < n_ops; ++j) {
+        const LinearArgs& a = ops[j];
+        const bool dual = a.W2 != nullptr;
+        if (a.m != m || !a.W || !a.Y || !a.xs || !a.partial || !a.tickets) return CSD_ERR_INVALID_ARG;
+        if (j == 0 && !a.xs_ready) return CSD_ERR_INVALID_ARG;
+        if (!tc_supported(a.m, a.N, a.K, dual)) return CSD_ERR_UNSUPPORTED;
+        if (dual != (a.epilogue == EPI_SWIGLU || a.epilogue == EPI_GEGLU)) return CSD_ERR_INVALID_ARG;
+        ChainOpDev& o = cp.op[j];
+        o.tiles = (a.N + TILE_N - 1) / TILE_N;
+        o.nkb = (a.K + KB - 1) / KB;
+        if ((long long)o.tiles * o.nkb * (dual ? 2 : 1) * (grid + 1) >= (1LL << 31)) return CSD_ERR_UNSUPPORTED;
+        if (!tensor_map_2d(a.W, a.N, a.K, TILE_N, &o.tmW)) return CSD_ERR_UNSUPPORTED;
+        o.tmW2 = o.tmW;
+        if (dual && !tensor_map_2d(a.W2, a.N, a.K, TILE_N, &o.tmW2)) return CSD_ERR_UNSUPPORTED;
+        if (!tensor_map_2d(a.xs, 3 * m, a.K, npad, &o.tmX)) return CSD_ERR_UNSUPPORTED;
+        o.Y = a.Y; o.ssq_in = a.gain ? a.ssq : nullptr; o.ssq_cnt = a.ssq_cnt;
+        o.out_xs = a.out_xs; o.out_gain = a.out_gain; o.out_ssq = a.out_ssq; o.out_ld = a.out_ld;
+        o.tickets = ops[0].tickets + ticket_off;
+        ticket_off += (size_t)o.tiles;
+        o.N = a.N; o.K = a.K; o.ldy = a.ldy; o.epilogue = a.epilogue; o.dual = dual ? 1 : 0; o.eps = a.eps;
+    }
+    cp.partial = ops[0].partial;
+    cp.done = done_dev;
+    cp.status = status_word_device();
+    *epoch_host += 1;
+    cp.done_target = *epoch_host * (unsigned)grid;
+    cp.n_ops = n_ops;
+    const size_t stage = (size_t)STAGE_BYTES + (size_t)npad * 128;
+    int stages = (int)((CHAIN_SMEM - 2048) / stage);
+    if (stages > 12) stages = 12;
+    cp.stages = stages;
+    const size_t smem = (size_t)stages * stage + 2048 + 1024;
+#define CSD_CH_CASE(MM) case MM: return launch_chain_m<MM>(cp, grid, smem, st);
+    switch (m) {
+        CSD_CH_CASE(1) CSD_CH_CASE(2) CSD_CH_CASE(3) CSD_CH_CASE(4) CSD_CH_CASE(5) CSD_CH_CASE(6) CSD_CH_CASE(7)
+        CSD_CH_CASE(8) CSD_CH_CASE(9) CSD_CH_CASE(10) CSD_CH_CASE(11) CSD_CH_CASE(12) CSD_CH_CASE(13)
+        CSD_CH_CASE(14) CSD_CH_CASE(15) CSD_CH_CASE(16) CSD_CH_CASE(17)
+    }
+#undef CSD_CH_CASE
+    return CSD_ERR_INVALID_ARG;
+}
+
+}  // namespace csd
