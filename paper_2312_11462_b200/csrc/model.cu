@@ -290,7 +290,7 @@ static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, c
 // Needs every one of them on the tensor-core kernel and the attention output in three-term form.
 static bool chain_applies(const csd_model* M, int m, int l) {
     const csd_model_config& c = M->cfg;
-    if (c.arch != 0 || gemm_path() == 1) return false;
+    if (c.arch != 0 || gemm_path() == 1 || gemm_path() == 3) return false;
     const int d = c.d_model, di = M->di, ff = c.d_ff;
     const bool last = l + 1 == c.n_layers;
     if (!last) {
