@@ -115,15 +115,21 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
     volatile int* abort_flag = &ctl->abort_flag;
 
     // this CTA's share of every GEMM of the chain
-    unsigned u0[CHAIN_MAX_OPS], cnt[CHAIN_MAX_OPS], units[CHAIN_MAX_OPS];
+    // (a GEMM with fewer units than CTAs is shared among its first `eff` CTAs only, so that every
+    // CTA between two that share a tile holds a part of it: the fix-up counts on that)
+    unsigned u0[CHAIN_MAX_OPS], cnt[CHAIN_MAX_OPS], units[CHAIN_MAX_OPS], eff[CHAIN_MAX_OPS];
     int total = 0;
 #pragma unroll
     for (int j = 0; j < CHAIN_MAX_OPS; ++j) {
         u0[j] = cnt[j] = units[j] = 0;
+        eff[j] = 1;
         if (j < cp.n_ops) {
             units[j] = (unsigned)cp.op[j].tiles * (unsigned)cp.op[j].nkb * (cp.op[j].dual ? 2u : 1u);
-            u0[j] = ch_unit_begin(cta, units[j], ctas);
-            cnt[j] = ch_unit_begin(cta + 1, units[j], ctas) - u0[j];
+            eff[j] = units[j] < ctas ? units[j] : ctas;
+            if (cta < eff[j]) {
+                u0[j] = ch_unit_begin(cta, units[j], eff[j]);
+                cnt[j] = ch_unit_begin(cta + 1, units[j], eff[j]) - u0[j];
+            }
             total += (int)cnt[j];
         }
     }
@@ -157,7 +163,11 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
                 if (gx < gw) {
                     if (xop > dep_ok_upto) {
                         // GEMM xop reads what GEMM xop-1 wrote: has every CTA finished xop-1 ?
-                        if ((int)(ld_acquire(cp.done + (xop - 1)) - cp.done_target) >= 0) dep_ok_upto = xop;
+                        if ((int)(ld_acquire(cp.done + (xop - 1)) - cp.done_target) >= 0) {
+                            // the rows were written with ordinary stores; the loads below go through the async proxy
+                            asm volatile("fence.proxy.async.global;" ::: "memory");
+                            dep_ok_upto = xop;
+                        }
                     }
                     if (xop <= dep_ok_upto) {
                         const ChainOpDev& o = cp.op[xop];
@@ -280,8 +290,8 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
                         }
                     __threadfence();
                     asm volatile("bar.sync 1, 128;" ::: "memory");
-                    const int c_lo = ch_cta_of_unit((unsigned)tile * per_tile, units[j], ctas);
-                    const int c_hi = ch_cta_of_unit((unsigned)(tile + 1) * per_tile - 1, units[j], ctas);
+                    const int c_lo = ch_cta_of_unit((unsigned)tile * per_tile, units[j], eff[j]);
+                    const int c_hi = ch_cta_of_unit((unsigned)(tile + 1) * per_tile - 1, units[j], eff[j]);
                     if (et == 0) {
                         const unsigned old = atomicAdd(&o.tickets[tile], 1u);
                         ctl->last_flag = (old == (unsigned)(c_hi - c_lo));
@@ -297,7 +307,7 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
 #pragma unroll
                         for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
                     for (int c = c_lo; c <= c_hi; ++c) {
-                        const int slot = (int)(ch_unit_begin(c, units[j], ctas) / per_tile) == tile ? 0 : 1;
+                        const int slot = (int)(ch_unit_begin(c, units[j], eff[j]) / per_tile) == tile ? 0 : 1;
                         const float* src = cp.partial + ((size_t)c * 2 + slot) * 2 * M * TILE_N + col;
                         float part[2][M];
 #pragma unroll
@@ -328,7 +338,7 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
                     }
                     if (n < o.N) {
                         float* y = o.Y + (size_t)r * o.ldy + n;
-                        if (o.epilogue == EPI_ADD) val += *y;
+                        if (o.epilogue == EPI_ADD) val += __ldcg(y);      // may have been written by another CTA of this launch
                         *y = val;
                     } else {
                         val = 0.f;
@@ -358,6 +368,7 @@ gemm_chain_kernel(const __grid_constant__ ChainParams cp) {
             if (dead) break;
             // report this GEMM finished by this CTA (its own tiles and any fix-ups it performed)
             __threadfence();
+            asm volatile("fence.proxy.async.global;" ::: "memory");
             asm volatile("bar.sync 1, 128;" ::: "memory");
             if (et == 0) atomicAdd(cp.done + j, 1u);
         }
