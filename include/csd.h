@@ -141,9 +141,7 @@ csd_status csd_model_profile_read(csd_model* m, void* stream, csd_profile* out);
 size_t csd_linear_workspace_bytes(int m, int N, int K);
 /* Which kernel the contraction uses, process-wide: 0 = automatic choice per shape, 1 = the
  * CUDA-core kernel (128-bit streaming loads, fp32 FMA), 2 = the tensor-core kernel (TMA-staged
- * weights, tcgen05.mma with fp32 accumulators in tensor memory) wherever it applies (K >= 64),
- * with the GEMMs of a layer's tail chained into one persistent kernel, 3 = as 2 but one kernel
- * per GEMM.
+ * weights, tcgen05.mma with fp32 accumulators in tensor memory) wherever it applies (K >= 64).
  * Both give the same result up to fp32 summation order; the switch exists to measure them. */
 csd_status csd_set_gemm_path(int path);
 csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, int m, float* Y_dev,

@@ -332,7 +332,7 @@ bool linear_uses_tensor_cores(int m, int N, int K, bool dual) {
     const int path = gemm_path();
     // measured on the 7B layer shapes the tensor-core kernel wins at every m (a 5-row review forward
     // takes 4.0 ms against 5.2 ms, a 17-row one 5.5 ms against 15 ms); tiny matrices stay on the simpler kernel
-    return path != 1 && tc_supported(m, N, K, dual) && (path >= 2 || (long long)N * K >= AUTO_TC_MIN_WEIGHTS);
+    return path != 1 && tc_supported(m, N, K, dual) && (path == 2 || (long long)N * K >= AUTO_TC_MIN_WEIGHTS);
 }
 
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
@@ -367,7 +367,7 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
 using namespace csd;
 
 extern "C" csd_status csd_set_gemm_path(int path) {
-    if (path < 0 || path > 3) return CSD_ERR_INVALID_ARG;
+    if (path < 0 || path > 2) return CSD_ERR_INVALID_ARG;
     set_gemm_path(path);
     return CSD_OK;
 }

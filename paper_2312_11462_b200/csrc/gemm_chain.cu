@@ -55,9 +55,9 @@ __device__ __forceinline__ int ch_cta_of_unit(unsigned u, unsigned units, unsign
     while (c > 0 && ch_unit_begin(c, units, ctas) > u) --c;
     return (int)c;
 }
-__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {   // one poll, no spinning
+__device__ __forceinline__ bool mbar_test(uint64_t* bar, uint32_t parity) {   // one poll; test_wait never suspends the thread, so the other cursor keeps moving
     uint32_t ok;
-    asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+    asm volatile("{ .reg .pred p; mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
                  : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }

@@ -136,7 +136,7 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
-        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, chain_done, total;
+        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, total;
     size_t layer_kv, layer_x;
 };
 
@@ -165,7 +165,6 @@ static WsLayout ws_layout(const csd_model_config& c) {
     size_t keys = c.max_seq > c.max_enc_len ? c.max_seq : c.max_enc_len;
     L.attn_partial = put(attn_scratch_bytes((int)keys, (int)H, (int)Dh));
     L.attn_tickets = put(H * 4);
-    L.chain_done = put(64);
     const size_t kmax = d > di ? (d > ff ? d : ff) : (di > ff ? di : ff);
     L.xs_tmp = put(3 * R * kmax * 2);
     L.ssq_tmp = put((size_t)split_ssq_entries((int)kmax) * R * 4);
@@ -221,7 +220,7 @@ struct LinOpt {
 // One linear layer of the forward; all of them share the model's split scratch.
 static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat16* W2, int N, int K, const float* X,
                          int ldx, int m, const __nv_bfloat16* gain, float* Y, int ldy, int epi, cudaStream_t st,
-                         const LinOpt* o = nullptr, LinearArgs* only_fill = nullptr) {
+                         const LinOpt* o = nullptr) {
     LinearArgs a;
     a.W = W; a.W2 = W2; a.N = N; a.K = K; a.X = X; a.ldx = ldx; a.m = m; a.gain = gain; a.eps = M->cfg.norm_eps;
     a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.partial = M->gemm_partial; a.tickets = M->gemm_tickets;
@@ -233,7 +232,6 @@ static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat
         }
         a.out_xs = o->out_xs; a.out_ld = o->out_ld; a.out_gain = o->out_gain; a.out_ssq = o->out_ssq;
     }
-    if (only_fill) { *only_fill = a; return CSD_OK; }
     ProfScope ps(M, 0, st);
     if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
     return launch_linear(a, st);
@@ -283,49 +281,6 @@ static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, c
     if (hand_on) { down.out_xs = M->xs_x; down.out_ld = d; down.out_gain = next_gain; down.out_ssq = M->ssq_x; }
     if (x_out) *x_out = hand_on;
     return linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, X, d, EPI_ADD, st, &down);
-}
-
-// Decoder-only layer tail as ONE kernel: attention-output projection -> gated feed-forward -> down
-// projection -> the next layer's q|k|v projection (or the output head after the last layer).
-// Needs every one of them on the tensor-core kernel and the attention output in three-term form.
-static bool chain_applies(const csd_model* M, int m, int l) {
-    const csd_model_config& c = M->cfg;
-    if (c.arch != 0 || gemm_path() == 1 || gemm_path() == 3) return false;
-    const int d = c.d_model, di = M->di, ff = c.d_ff;
-    const bool last = l + 1 == c.n_layers;
-    if (!last) {
-        const LayerW& nx = M->dec[l + 1];
-        if (!(nx.wk == nx.wq + (size_t)di * d && nx.wv == nx.wk + (size_t)di * d)) return false;
-    }
-    return linear_uses_tensor_cores(m, d, di, false) && linear_uses_tensor_cores(m, ff, d, true) &&
-           linear_uses_tensor_cores(m, d, ff, false) &&
-           linear_uses_tensor_cores(m, last ? c.vocab : 3 * di, d, false);
-}
-
-static csd_status chain_layer_tail(csd_model* M, int l, int m, float* logits, cudaStream_t st) {
-    const csd_model_config& c = M->cfg;
-    const int d = c.d_model, di = M->di, ff = c.d_ff, cnt_d = 4 * ((d + 127) / 128);
-    const LayerW& y = M->dec[l];
-    const bool last = l + 1 == c.n_layers;
-    LinearArgs ops[4];
-    LinOpt o0, o1, o2, o3;
-    o0.xs_in = M->xs_attn; o0.out_xs = M->xs_x; o0.out_ld = d; o0.out_gain = y.norm2; o0.out_ssq = M->ssq_x;
-    linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st, &o0, &ops[0]);
-    o1.xs_in = M->xs_x; o1.ssq_in = M->ssq_x; o1.ssq_cnt = cnt_d; o1.out_xs = M->xs_act; o1.out_ld = ff;
-    linear(M, y.wgate, y.wup, ff, d, M->x, d, m, y.norm2, M->act, ff, c.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, st, &o1, &ops[1]);
-    o2.xs_in = M->xs_act; o2.out_xs = M->xs_x; o2.out_ld = d; o2.out_ssq = M->ssq_x;
-    o2.out_gain = last ? M->final_norm : M->dec[l + 1].norm1;
-    linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, M->x, d, EPI_ADD, st, &o2, &ops[2]);
-    o3.xs_in = M->xs_x; o3.ssq_in = M->ssq_x; o3.ssq_cnt = cnt_d;
-    if (last)
-        linear(M, M->lm_head, nullptr, c.vocab, d, M->x, d, m, M->final_norm, logits, c.vocab, EPI_STORE, st, &o3, &ops[3]);
-    else
-        linear(M, M->dec[l + 1].wq, nullptr, 3 * di, d, M->x, d, m, M->dec[l + 1].norm1, M->qkv, 3 * di, EPI_STORE, st,
-               &o3, &ops[3]);
-    ProfScope ps(M, 0, st);
-    if (M->prof)
-        for (int j = 0; j < 4; ++j) M->prof_gemm_bytes += (double)ops[j].N * ops[j].K * 2.0 * (ops[j].W2 ? 2.0 : 1.0);
-    return launch_linear_chain(ops, 4, M->chain_done, &M->chain_epoch, st);
 }
 
 }  // namespace csd
@@ -385,7 +340,6 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     M->act = (float*)(ws + L.act);
     M->gemm_partial = (float*)(ws + L.gemm_partial); M->gemm_tickets = (unsigned*)(ws + L.gemm_tickets);
     M->xs_tmp = (__nv_bfloat16*)(ws + L.xs_tmp); M->ssq_tmp = (float*)(ws + L.ssq_tmp);
-    M->chain_done = (unsigned*)(ws + L.chain_done);
     M->xs_x = (__nv_bfloat16*)(ws + L.xs_x); M->xs_attn = (__nv_bfloat16*)(ws + L.xs_attn);
     M->xs_act = (__nv_bfloat16*)(ws + L.xs_act); M->ssq_x = (float*)(ws + L.ssq_x);
     M->attn_partial = (float*)(ws + L.attn_partial); M->attn_tickets = (unsigned*)(ws + L.attn_tickets);
@@ -393,7 +347,6 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.attn_partial - L.gemm_tickets, st);
     if (e == cudaSuccess) e = cudaMemsetAsync(ws + L.attn_tickets, 0, (size_t)cfg->n_heads * 4, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(ws + L.chain_done, 0, 64, st);
     if (e != cudaSuccess) { delete M; return note_cuda(e); }
     if (cfg->arch == 0) {
         M->rope_c = (float*)(ws + L.rope_c); M->rope_s = (float*)(ws + L.rope_s);
@@ -529,19 +482,18 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
     }
     // x_ready: M->xs_x / M->ssq_x hold the residual rows (times the gain of the norm that reads them
     // next) in three-term form, written by the epilogue of the GEMM that produced the rows
-    bool x_ready = false, qkv_done = false, head_done = false;
+    bool x_ready = false;
     const int ff = c.d_ff, cnt_d = 4 * ((d + 127) / 128);
     const bool tc_o = linear_uses_tensor_cores(m, d, di, false);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& y = M->dec[l];
         __nv_bfloat16* Kl = M->kcache + (size_t)l * M->layer_kv;
         __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
-        if (!qkv_done) {
+        {
             LinOpt qo;
             if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = cnt_d; }
             CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         }
-        qkv_done = false;
         {
             ProfScope ps(M, 2, st);
             PdlLaunch L(dim3(m, H), dim3(64), 0, st);
@@ -557,12 +509,6 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         a.out = M->attn; a.ldo = di; a.partial = M->attn_partial; a.tickets = M->attn_tickets;
         if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
         CSD_TRY(attention(M, a, st));
-        if (chain_applies(M, m, l)) {    // the rest of the layer and the next projection in one kernel
-            CSD_TRY(chain_layer_tail(M, l, m, logits_out_dev, st));
-            x_ready = true;
-            if (l + 1 == c.n_layers) head_done = true; else qkv_done = true;
-            continue;
-        }
         // output projection into the residual rows; hands them on to the norm that follows
         LinOpt oo;
         if (tc_o) oo.xs_in = M->xs_attn;
@@ -597,7 +543,6 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
     }
     LinOpt ho;
     if (x_ready) { ho.xs_in = M->xs_x; ho.ssq_in = M->ssq_x; ho.ssq_cnt = cnt_d; }
-    if (!head_done)
     CSD_TRY(linear(M, M->lm_head, nullptr, V, d, M->x, d, m, M->final_norm, logits_out_dev, V, EPI_STORE, st, &ho));
     CSD_CUDA(cudaGetLastError());
     return CSD_OK;
