@@ -239,7 +239,7 @@ def run_ours(args):
     review_gbs = (weight_bytes + kv_bytes) / (review_us * 1e-6) / 1e9
     gemm_launch_us = 1e3 * prof["gemm_ms"] / max(prof["gemm_launches"], 1)
     gemm_gbs = prof["gemm_weight_bytes"] / (prof["gemm_ms"] * 1e-3) / 1e9
-    roofline = {"bound": "hbm", "kernel": "skinny_gemm_kernel (weight-streaming GEMM, m=5)", "achieved": gemm_gbs,
+    roofline = {"bound": "hbm", "kernel": "skinny_gemm_tc_kernel (TMA-staged weight-streaming GEMM on tcgen05, m=5)", "achieved": gemm_gbs,
                 "peak": peak, "peak_kind": f"{peak_kind} STREAM-style copy", "unit": "GB/s", "frac": gemm_gbs / peak,
                 "traffic": None, "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
                 "us_per_launch": gemm_launch_us}
@@ -272,6 +272,39 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_review_only(args):
+    """Profiling aid: `--review-only N` runs N review forwards (m = k+1 = 5 rows over a committed
+    128-token cache) of the 7B-shaped target, optionally cut to `--layers L` layers so that a
+    counter capture holds a few GB at most, then one accept call, and prints their mean times."""
+    import torch
+    import workloads
+    from dataclasses import replace
+    from paper_2312_11462_b200 import binding as b
+    ts = workloads.SHAPES["llama7b"]
+    if args.layers:
+        ts = replace(ts, n_layers=args.layers)
+    tb = workloads.make_weights(ts, seed=100, device="cuda")
+    prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, PROMPT_LEN + MAX_BLOCK + 1, seed=1000)).cuda()
+    target = b.Model(ts, tb)
+    for p0 in range(0, PROMPT_LEN, 16):
+        target.csd_review_forward(prompt[p0:p0 + 16], p0)
+    blk = prompt[PROMPT_LEN:PROMPT_LEN + MAX_BLOCK + 1].contiguous()
+    logits = torch.empty(MAX_BLOCK + 1, ts.vocab, device="cuda")
+    ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    ev0.record()
+    for _ in range(args.review_only):
+        target.csd_review_forward(blk, PROMPT_LEN, logits)
+    ev1.record()
+    torch.cuda.synchronize()
+    tok = blk[:MAX_BLOCK].reshape(1, MAX_BLOCK).contiguous()
+    n_acc, out = b.csd_spec_accept(logits.reshape(1, MAX_BLOCK + 1, ts.vocab), None, tok, 0.0)
+    torch.cuda.synchronize()
+    print(json.dumps({"review_only": args.review_only, "layers": ts.n_layers,
+                      "review_us": 1e3 * ev0.elapsed_time(ev1) / args.review_only,
+                      "n_acc": int(n_acc[0]), "out": int(out[0])}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -279,8 +312,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--review-only", type=int, default=0, help="profiling aid: only N review forwards of the target")
+    ap.add_argument("--layers", type=int, default=0, help="with --review-only: cut the target to L layers")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.review_only:
+        run_review_only(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
