@@ -1,36 +1,54 @@
 // Attention of a block of m <= 17 query rows against a bf16 K/V cache, split along the keys.
 //
-// grid = (heads, splits).  A CTA walks its key range in tiles of 64 positions staged in shared
-// memory, keeps an online softmax per row (running max, running sum, rescaled accumulator) and
-// leaves (max, sum, unnormalised output) in scratch; the CTA that arrives last at the head's
-// ticket merges the splits.  Rows see keys [0, n_keys + r] when causal (the drafted block is
-// causal inside itself), all n_keys otherwise (cross-attention, encoder).
+// grid = (heads, splits), the splits of one head forming a thread-block cluster.  A CTA walks its
+// key range in tiles of 64 positions: thread 0 requests each tile's committed rows with two bulk
+// copies (a head's rows are contiguous in the cache) that complete on an mbarrier, two tiles in
+// flight; the block's own rows (self-attention of a drafted block) are rotated, rounded to bf16,
+// written to the cache and laid over the staged tile by the CTA whose range holds them, so the
+// separate append pass and its round trip through HBM are gone.  Every CTA keeps an online softmax
+// per row (running max, running sum, rescaled accumulator); the splits then exchange (max, sum,
+// unnormalised output) through distributed shared memory and each merges a slice of the output.
+// Rows see keys [0, n_keys + r) when causal, all n_keys otherwise (cross-attention, encoder).
+#include <cooperative_groups.h>
 #include "attention.cuh"
+#include "tc_common.cuh"
+
+namespace cg = cooperative_groups;
 
 namespace csd {
 
 constexpr int AT = 256;
 constexpr int TILE = 64;
 constexpr int MAXM = CSD_MAX_ROWS;
-constexpr int MAX_SPLITS = 32;
+constexpr int MAX_SPLITS = 8;          // portable cluster size
+constexpr int STAGES = 2;
 
 template <int DH> struct AttnCfg {
-    static constexpr int KROW = DH + (DH == 32 ? 0 : 32);   // bf16 elements per staged row (bank spread)
     static constexpr int HP = DH / 2;                        // dim pairs
     static constexpr int G = AT / HP;                        // row groups in the PV phase
     static constexpr int RG = (MAXM + G - 1) / G;            // rows per group
     static constexpr int NC = DH / 32;                       // 8-element chunks per score thread
-    static constexpr size_t SMEM = (size_t)2 * TILE * KROW * 2 + (size_t)MAXM * DH * 4 + (size_t)MAXM * TILE * 4 +
-                                   3 * 32 * 4;
+    static constexpr int QROW = NC * 36;                     // q row: 32-float groups, 4 floats of skew each
+    static constexpr int REC = DH + 2;                       // merge record: output row, max, sum
+    static constexpr size_t TILE_BYTES = (size_t)TILE * DH * 2;
+    static constexpr size_t QS_FLOATS = (size_t)MAXM * (QROW > REC ? QROW : REC);
+    static constexpr size_t SMEM = 2 * STAGES * TILE_BYTES + QS_FLOATS * 4 + (size_t)MAXM * TILE * 4 +
+                                   2 * (size_t)MAXM * DH * 2 + 3 * 32 * 4 + 128;
 };
 
 struct AttnParams {
-    const float* q; const __nv_bfloat16* Kc; const __nv_bfloat16* Vc; const float* bias; float* out;
+    const float* q; const float* k_new; const float* v_new; const float* rope_cos; const float* rope_sin;
+    __nv_bfloat16* Kc; __nv_bfloat16* Vc; const float* bias; float* out;
     __nv_bfloat16* out_xs; int out_xs_ld;
-    float* partial; unsigned* tickets;
-    int ldq, m, cap, H, n_keys, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
+    int* status;
+    int ldq, ld_new, m, cap, H, n_keys, n_old, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
 };
+
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_u32(dst)), "l"(src), "r"(bytes), "r"(smem_u32(bar)) : "memory");
+}
 
 // two neighbouring output columns of row r as three bf16 terms each (rows term * m + r)
 __device__ __forceinline__ void store_split(__nv_bfloat16* xs, int ld, int m, int r, int col, float a, float b) {
@@ -47,63 +65,125 @@ template <int DH>
 __global__ void __launch_bounds__(AT)
 block_attention_kernel(const AttnParams p) {
     using C = AttnCfg<DH>;
-    extern __shared__ __align__(16) unsigned char smem_raw[];
-    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem_raw);
-    __nv_bfloat16* Vs = Ks + TILE * C::KROW;
-    float* qs = reinterpret_cast<float*>(Vs + TILE * C::KROW);   // [MAXM][DH]
-    float* sc = qs + MAXM * DH;                                  // [MAXM][TILE]
-    float* row_m = sc + MAXM * TILE;                             // [32]
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __nv_bfloat16* Ks = reinterpret_cast<__nv_bfloat16*>(smem_raw);            // [STAGES][TILE][DH]
+    __nv_bfloat16* Vs = Ks + STAGES * TILE * DH;
+    float* qs = reinterpret_cast<float*>(Vs + STAGES * TILE * DH);            // [MAXM][QROW]; later [MAXM][REC]
+    float* sc = qs + C::QS_FLOATS;                                            // [MAXM][TILE]
+    __nv_bfloat16* newK = reinterpret_cast<__nv_bfloat16*>(sc + MAXM * TILE); // [MAXM][DH] the block's own rows
+    __nv_bfloat16* newV = newK + MAXM * DH;
+    float* row_m = reinterpret_cast<float*>(newV + MAXM * DH);                // [32]
     float* row_l = row_m + 32;
     float* row_a = row_l + 32;
-    __shared__ int s_last;
+    uint64_t* full = reinterpret_cast<uint64_t*>(row_a + 32);                 // [STAGES]
 
+    cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, split = blockIdx.y;
-    const int m = p.m;
+    const int m = p.m, half = DH / 2;
     const int total = p.causal ? p.n_keys + m - 1 : p.n_keys;   // keys any row may see
     const int s_begin = split * p.split_len;
     const int s_end = min(total, s_begin + p.split_len);
+    const int n_tiles = s_end > s_begin ? (s_end - s_begin + TILE - 1) / TILE : 0;
+    __nv_bfloat16* Kh = p.Kc + (size_t)h * p.cap * DH;
+    __nv_bfloat16* Vh = p.Vc + (size_t)h * p.cap * DH;
+    const float* bias_h = p.bias ? p.bias + (size_t)h * p.bias_len : nullptr;
 
-    pdl_wait();       // q and the appended K/V rows come from the kernels before this one
-    pdl_trigger();
-    for (int i = tid; i < m * DH; i += AT) qs[i] = p.q[(size_t)(i / DH) * p.ldq + h * DH + (i % DH)];
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
     if (tid < 32) { row_m[tid] = -INFINITY; row_l[tid] = 0.f; row_a[tid] = 1.f; }
+    __syncthreads();
+
+    pdl_wait();       // q, the block's k and v rows and every committed cache row come from earlier kernels
+    pdl_trigger();
+
+    // committed rows of tile `it` (the rest of the tile, if any, are the block's own rows)
+    auto old_rows = [&](int it) {
+        const int t0 = s_begin + it * TILE;
+        return max(0, min(min(t0 + TILE, s_end), p.n_old) - t0);
+    };
+    auto request = [&](int it) {
+        const int st = it % STAGES, t0 = s_begin + it * TILE, cnt = old_rows(it);
+        if (cnt <= 0) return;
+        const uint32_t bytes = (uint32_t)cnt * DH * 2;
+        mbar_expect_tx(&full[st], 2 * bytes);
+        bulk_load(Ks + (size_t)st * TILE * DH, Kh + (size_t)t0 * DH, bytes, &full[st]);
+        bulk_load(Vs + (size_t)st * TILE * DH, Vh + (size_t)t0 * DH, bytes, &full[st]);
+    };
+    if (tid == 0)
+        for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
+
+    // ---- the block's rows: q (rotated) into shared memory; k (rotated) and v rounded to bf16, kept
+    //      for the tiles that hold them and written to the cache by the CTA whose range they fall in
+    for (int i = tid; i < m * half; i += AT) {
+        const int r = i / half, d = i % half, pos = p.n_old + r;
+        float c = 1.f, s = 0.f;
+        if (p.rope_cos) { c = p.rope_cos[(size_t)pos * half + d]; s = p.rope_sin[(size_t)pos * half + d]; }
+        const float* qr = p.q + (size_t)r * p.ldq + h * DH;
+        const float q0 = qr[d], q1 = qr[d + half];
+        const int e0 = d, e1 = d + half;
+        qs[r * C::QROW + (e0 >> 5) * 36 + (e0 & 31)] = q0 * c - q1 * s;
+        qs[r * C::QROW + (e1 >> 5) * 36 + (e1 & 31)] = q0 * s + q1 * c;
+        if (p.k_new) {
+            const float* kr = p.k_new + (size_t)r * p.ld_new + h * DH;
+            const float* vr = p.v_new + (size_t)r * p.ld_new + h * DH;
+            const float k0 = kr[d], k1 = kr[d + half];
+            const __nv_bfloat16 ka = __float2bfloat16_rn(k0 * c - k1 * s), kb = __float2bfloat16_rn(k0 * s + k1 * c);
+            const __nv_bfloat16 va = __float2bfloat16_rn(vr[d]), vb = __float2bfloat16_rn(vr[d + half]);
+            newK[r * DH + d] = ka; newK[r * DH + d + half] = kb;
+            newV[r * DH + d] = va; newV[r * DH + d + half] = vb;
+            if (pos >= s_begin && pos < s_end) {
+                Kh[(size_t)pos * DH + d] = ka; Kh[(size_t)pos * DH + d + half] = kb;
+                Vh[(size_t)pos * DH + d] = va; Vh[(size_t)pos * DH + d + half] = vb;
+            }
+        }
+    }
 
     const int dp = tid % C::HP, g = tid / C::HP;
     float acc[C::RG][2];
 #pragma unroll
     for (int rr = 0; rr < C::RG; ++rr) { acc[rr][0] = 0.f; acc[rr][1] = 0.f; }
 
-    const __nv_bfloat16* Kh = p.Kc + (size_t)h * p.cap * DH;
-    const __nv_bfloat16* Vh = p.Vc + (size_t)h * p.cap * DH;
-    const float* bias_h = p.bias ? p.bias + (size_t)h * p.bias_len : nullptr;
-
-    for (int t0 = s_begin; t0 < s_end; t0 += TILE) {
-        __syncthreads();   // previous tile fully consumed (also orders the qs / row state set-up)
-        for (int idx = tid; idx < TILE * (DH / 8); idx += AT) {
-            const int j = idx / (DH / 8), c = idx % (DH / 8);
-            uint4 kv = make_uint4(0, 0, 0, 0), vv = make_uint4(0, 0, 0, 0);
-            if (t0 + j < s_end) {
-                kv = *reinterpret_cast<const uint4*>(Kh + (size_t)(t0 + j) * DH + c * 8);
-                vv = *reinterpret_cast<const uint4*>(Vh + (size_t)(t0 + j) * DH + c * 8);
+    bool failed = false;
+    for (int it = 0; it < n_tiles; ++it) {
+        const int st = it % STAGES, t0 = s_begin + it * TILE;
+        const int ok = old_rows(it) <= 0 || mbar_wait(&full[st], (uint32_t)(it / STAGES) & 1u);
+        if (__syncthreads_or(!ok)) {      // (also orders the set-up above before the first tile)
+            if (!ok) mbar_wait(&full[st], (uint32_t)(it / STAGES) & 1u);   // once more, so no copy is in flight at exit
+            failed = true;
+            break;
+        }
+        __nv_bfloat16* Kt = Ks + (size_t)st * TILE * DH;
+        __nv_bfloat16* Vt = Vs + (size_t)st * TILE * DH;
+        const int valid = min(TILE, s_end - t0);
+        {   // lay the block's own rows over the tile; clear the value rows past the end of the range
+            const int new_lo = max(t0, p.n_old), n_new = t0 + valid - new_lo;
+            for (int idx = tid; idx < n_new * (DH / 8); idx += AT) {
+                const int row = idx / (DH / 8), c = idx % (DH / 8), j = new_lo + row - t0, r = new_lo + row - p.n_old;
+                *reinterpret_cast<uint4*>(Kt + j * DH + c * 8) = *reinterpret_cast<const uint4*>(newK + r * DH + c * 8);
+                *reinterpret_cast<uint4*>(Vt + j * DH + c * 8) = *reinterpret_cast<const uint4*>(newV + r * DH + c * 8);
             }
-            *reinterpret_cast<uint4*>(Ks + j * C::KROW + c * 8) = kv;
-            *reinterpret_cast<uint4*>(Vs + j * C::KROW + c * 8) = vv;
+            for (int idx = tid; idx < (TILE - valid) * (DH / 8); idx += AT)
+                *reinterpret_cast<uint4*>(Vt + (size_t)valid * DH + idx * 8) = make_uint4(0, 0, 0, 0);
         }
         __syncthreads();
-        // ---- scores: 4 threads per key, each over a quarter of the head dimension
+        // ---- scores: 4 threads per key, each over a quarter of the head dimension.  The 32-element
+        //      group a thread reads at step c is rotated by the key index, so that neighbouring keys
+        //      (whose rows start a multiple of 128 bytes apart) hit different banks.
         {
             const int j = tid >> 2, part = tid & 3;
             uint4 kreg[C::NC];
 #pragma unroll
             for (int c = 0; c < C::NC; ++c)
-                kreg[c] = *reinterpret_cast<const uint4*>(Ks + j * C::KROW + (c * 4 + part) * 8);
+                kreg[c] = *reinterpret_cast<const uint4*>(Kt + j * DH + (((c + j) % C::NC) * 4 + part) * 8);
             const int key = t0 + j;
             for (int r = 0; r < m; ++r) {
                 float d = 0.f;
 #pragma unroll
                 for (int c = 0; c < C::NC; ++c) {
-                    const float* qp = qs + r * DH + (c * 4 + part) * 8;
+                    const float* qp = qs + r * C::QROW + ((c + j) % C::NC) * 36 + part * 8;
                     const float4 qa = *reinterpret_cast<const float4*>(qp);
                     const float4 qb = *reinterpret_cast<const float4*>(qp + 4);
                     d = fmaf(bf16lo(kreg[c].x), qa.x, d); d = fmaf(bf16hi(kreg[c].x), qa.y, d);
@@ -161,7 +241,7 @@ block_attention_kernel(const AttnParams p) {
             float v[4][2];
 #pragma unroll
             for (int i = 0; i < 4; ++i) {
-                const uint32_t w = *reinterpret_cast<const uint32_t*>(Vs + (j4 + i) * C::KROW + 2 * dp);
+                const uint32_t w = *reinterpret_cast<const uint32_t*>(Vt + (j4 + i) * DH + 2 * dp);
                 v[i][0] = bf16lo(w); v[i][1] = bf16hi(w);
             }
 #pragma unroll
@@ -176,8 +256,13 @@ block_attention_kernel(const AttnParams p) {
                 }
             }
         }
+        __syncthreads();           // tile consumed: its stage may be filled again
+        if (tid == 0 && it + STAGES < n_tiles) {
+            fence_async_smem();    // the overlay above wrote this stage through the generic proxy
+            request(it + STAGES);
+        }
     }
-    __syncthreads();
+    if (failed && tid == 0) set_status(p.status, CSD_ERR_TIMEOUT);
 
     if (p.nsplit == 1) {
 #pragma unroll
@@ -192,41 +277,31 @@ block_attention_kernel(const AttnParams p) {
         }
         return;
     }
-    // ---- leave this split's partial result, last arrival merges
-    constexpr int REC = DH + 2;
-    float* mine = p.partial + ((size_t)h * p.nsplit + split) * MAXM * REC;
+    // ---- leave this split's (output, max, sum) in shared memory; after the cluster barrier every
+    //      CTA of the head merges its share of the output elements from all the splits' records
+    float* rec = qs;      // the q rows are not needed any more (all threads are past the last tile)
 #pragma unroll
     for (int rr = 0; rr < C::RG; ++rr) {
         const int r = g + rr * C::G;
         if (r < m) {
-            mine[r * REC + 2 * dp] = acc[rr][0];
-            mine[r * REC + 2 * dp + 1] = acc[rr][1];
+            rec[r * C::REC + 2 * dp] = acc[rr][0];
+            rec[r * C::REC + 2 * dp + 1] = acc[rr][1];
         }
     }
-    if (tid < m) { mine[tid * REC + DH] = row_m[tid]; mine[tid * REC + DH + 1] = row_l[tid]; }
-    __threadfence();
-    __syncthreads();
-    if (tid == 0) {
-        unsigned old = atomicAdd(&p.tickets[h], 1u);
-        s_last = (old == (unsigned)p.nsplit - 1u);
-        if (s_last) p.tickets[h] = 0u;
-    }
-    __syncthreads();
-    if (!s_last) return;
-    __threadfence();
-    const float* all = p.partial + (size_t)h * p.nsplit * MAXM * REC;
-    for (int i = tid; i < m * DH; i += AT) {
+    if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
+    cluster.sync();
+    for (int i = split * AT + tid; i < m * DH; i += p.nsplit * AT) {
         const int r = i / DH, d = i % DH;
         float M = -INFINITY;
-        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, __ldcg(all + ((size_t)s * MAXM + r) * REC + DH));
+        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(rec, s)[r * C::REC + DH]);
         float num = 0.f, den = 0.f;
         for (int s = 0; s < p.nsplit; ++s) {
-            const float* rec = all + ((size_t)s * MAXM + r) * REC;
-            const float ms = __ldcg(rec + DH);
+            const float* rs = cluster.map_shared_rank(rec, s) + r * C::REC;
+            const float ms = rs[DH];
             if (ms > -INFINITY) {
                 const float w = expf(ms - M);
-                num = fmaf(__ldcg(rec + d), w, num);
-                den = fmaf(__ldcg(rec + DH + 1), w, den);
+                num = fmaf(rs[d], w, num);
+                den = fmaf(rs[DH + 1], w, den);
             }
         }
         const float o = den > 0.f ? num / den : 0.f;
@@ -240,10 +315,12 @@ block_attention_kernel(const AttnParams p) {
             xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
         }
     }
+    cluster.sync();       // no CTA leaves while another may still read its record
 }
 
-// One 64-key tile per CTA while that still gives no more than about two CTAs per SM: short caches
-// are latency-bound, and a CTA that walks several tiles pays one round trip per tile.
+// One 64-key tile per CTA while that keeps the splits of a head inside one portable cluster (8)
+// and the grid near two CTAs per SM: short caches are latency-bound, and more splits mean more
+// tiles in flight at once; long caches walk several tiles per CTA, two requests ahead.
 int attn_splits(int total_keys, int H) {
     int by_sm = (2 * 148 + H - 1) / H;
     int by_len = (total_keys + TILE - 1) / TILE;
@@ -251,11 +328,6 @@ int attn_splits(int total_keys, int H) {
     if (n < 1) n = 1;
     if (n > MAX_SPLITS) n = MAX_SPLITS;
     return n;
-}
-
-size_t attn_scratch_bytes(int max_keys, int H, int Dh) {
-    (void)max_keys;
-    return align_up((size_t)H * MAX_SPLITS * MAXM * (Dh + 2) * sizeof(float), 256);
 }
 
 template <int DH>
@@ -266,8 +338,19 @@ static csd_status launch_dh(const AttnParams& ap, cudaStream_t st) {
         CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnCfg<DH>::SMEM));
         attr_set = true;
     }
-    PdlLaunch L(dim3((unsigned)ap.H, (unsigned)ap.nsplit), dim3(AT), AttnCfg<DH>::SMEM, st);
-    CSD_CUDA(cudaLaunchKernelEx(&L.cfg, kern, ap));
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3((unsigned)ap.H, (unsigned)ap.nsplit);
+    cfg.blockDim = dim3(AT);
+    cfg.dynamicSmemBytes = AttnCfg<DH>::SMEM;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // the splits of one head exchange results on chip
+    attr[1].val.clusterDim.x = 1; attr[1].val.clusterDim.y = (unsigned)ap.nsplit; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, ap));
     count_launch();
     return CSD_OK;
 }
@@ -275,18 +358,24 @@ static csd_status launch_dh(const AttnParams& ap, cudaStream_t st) {
 csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     if (!a.q || !a.Kc || !a.Vc || !a.out || a.m < 1 || a.m > MAXM || a.H < 1 || a.n_keys < 0)
         return CSD_ERR_INVALID_ARG;
+    const bool append = a.k_new != nullptr;
+    if (append && (!a.v_new || !a.causal || a.n_keys < 1)) return CSD_ERR_INVALID_ARG;
+    if ((a.rope_cos != nullptr) != (a.rope_sin != nullptr) || (a.rope_cos && !append)) return CSD_ERR_INVALID_ARG;
+    if ((((uintptr_t)a.Kc) & 15) || (((uintptr_t)a.Vc) & 15)) return CSD_ERR_INVALID_ARG;
     const int total = a.causal ? a.n_keys + a.m - 1 : a.n_keys;
     if (total < 1 || total > a.cap) return CSD_ERR_CAPACITY;
     AttnParams ap;
-    ap.q = a.q; ap.Kc = a.Kc; ap.Vc = a.Vc; ap.bias = a.bias; ap.out = a.out; ap.partial = a.partial;
-    ap.tickets = a.tickets; ap.ldq = a.ldq; ap.m = a.m; ap.cap = a.cap; ap.H = a.H; ap.n_keys = a.n_keys;
+    ap.q = a.q; ap.k_new = a.k_new; ap.v_new = a.v_new; ap.ld_new = a.ld_new; ap.rope_cos = a.rope_cos;
+    ap.rope_sin = a.rope_sin; ap.Kc = a.Kc; ap.Vc = a.Vc; ap.bias = a.bias; ap.out = a.out;
+    ap.status = status_word_device();
+    ap.ldq = a.ldq; ap.m = a.m; ap.cap = a.cap; ap.H = a.H; ap.n_keys = a.n_keys;
+    ap.n_old = append ? a.n_keys - 1 : total;
     ap.causal = a.causal; ap.bias_len = a.bias_len; ap.bias_zero = a.bias_zero; ap.q_pos0 = a.q_pos0;
     ap.ldo = a.ldo; ap.scale = a.scale; ap.out_xs = a.out_xs; ap.out_xs_ld = a.out_xs_ld;
     ap.nsplit = attn_splits(total, a.H);
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;
     ap.nsplit = (total + ap.split_len - 1) / ap.split_len;
-    if (ap.nsplit > 1 && (!a.partial || !a.tickets)) return CSD_ERR_INVALID_ARG;
     switch (a.Dh) {
         case 32: return launch_dh<32>(ap, st);
         case 64: return launch_dh<64>(ap, st);

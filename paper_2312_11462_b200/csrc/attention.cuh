@@ -7,8 +7,8 @@ namespace csd {
 struct AttnArgs {
     const float* q = nullptr;             // [m, ldq] fp32; head h occupies columns h*Dh .. h*Dh+Dh-1
     int ldq = 0, m = 0;
-    const __nv_bfloat16* Kc = nullptr;    // [H][cap][Dh]
-    const __nv_bfloat16* Vc = nullptr;
+    __nv_bfloat16* Kc = nullptr;          // [H][cap][Dh]
+    __nv_bfloat16* Vc = nullptr;
     int cap = 0, H = 0, Dh = 0;
     int n_keys = 0;                       // keys visible to row 0 (causal: row r sees n_keys + r)
     int causal = 0;
@@ -20,13 +20,18 @@ struct AttnArgs {
     int ldo = 0;
     __nv_bfloat16* out_xs = nullptr;      // optional: the output rows as three bf16 terms, row = term * m + r
     int out_xs_ld = 0;
-    float* partial = nullptr;             // split scratch (attn_scratch_bytes)
-    unsigned* tickets = nullptr;          // H zero-initialised words
-    int max_keys = 0;                     // capacity used to size the scratch
+    // Self-attention of a drafted block (causal, n_keys = committed keys + 1): the block's own key
+    // and value rows are still fp32 projections [m, ld_new]; the kernel rotates q and k (when
+    // rope tables [pos][Dh/2] are given), rounds k and v to bf16, appends them to the cache at
+    // positions n_keys-1 .. n_keys+m-2 and attends over committed and new rows alike.
+    const float* k_new = nullptr;
+    const float* v_new = nullptr;
+    int ld_new = 0;
+    const float* rope_cos = nullptr;
+    const float* rope_sin = nullptr;
 };
 
 int attn_splits(int total_keys, int H);
-size_t attn_scratch_bytes(int max_keys, int H, int Dh);
 csd_status launch_attention(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace csd

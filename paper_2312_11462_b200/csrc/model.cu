@@ -136,7 +136,7 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
-        buckets, gemm_partial, gemm_tickets, attn_partial, attn_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, total;
+        buckets, gemm_partial, gemm_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, total;
     size_t layer_kv, layer_x;
 };
 
@@ -162,9 +162,6 @@ static WsLayout ws_layout(const csd_model_config& c) {
     mat(3 * di, d, false); mat(di, d, false); mat(d, di, false); mat(ff, d, true); mat(d, ff, false); mat(V, d, false);
     L.gemm_partial = put(gp);
     L.gemm_tickets = put((size_t)linear_ticket_count((int)nmax) * 4);
-    size_t keys = c.max_seq > c.max_enc_len ? c.max_seq : c.max_enc_len;
-    L.attn_partial = put(attn_scratch_bytes((int)keys, (int)H, (int)Dh));
-    L.attn_tickets = put(H * 4);
     const size_t kmax = d > di ? (d > ff ? d : ff) : (di > ff ? di : ff);
     L.xs_tmp = put(3 * R * kmax * 2);
     L.ssq_tmp = put((size_t)split_ssq_entries((int)kmax) * R * 4);
@@ -342,11 +339,9 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     M->xs_tmp = (__nv_bfloat16*)(ws + L.xs_tmp); M->ssq_tmp = (float*)(ws + L.ssq_tmp);
     M->xs_x = (__nv_bfloat16*)(ws + L.xs_x); M->xs_attn = (__nv_bfloat16*)(ws + L.xs_attn);
     M->xs_act = (__nv_bfloat16*)(ws + L.xs_act); M->ssq_x = (float*)(ws + L.ssq_x);
-    M->attn_partial = (float*)(ws + L.attn_partial); M->attn_tickets = (unsigned*)(ws + L.attn_tickets);
     M->status = status;
     cudaStream_t st = (cudaStream_t)stream;
-    cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.attn_partial - L.gemm_tickets, st);
-    if (e == cudaSuccess) e = cudaMemsetAsync(ws + L.attn_tickets, 0, (size_t)cfg->n_heads * 4, st);
+    cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.xs_tmp - L.gemm_tickets, st);
     if (e != cudaSuccess) { delete M; return note_cuda(e); }
     if (cfg->arch == 0) {
         M->rope_c = (float*)(ws + L.rope_c); M->rope_s = (float*)(ws + L.rope_s);
@@ -440,7 +435,6 @@ extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_token
             a.q = M->qkv_enc + (size_t)r0 * 3 * di; a.ldq = 3 * di; a.m = m; a.Kc = M->ek; a.Vc = M->ev; a.cap = E;
             a.H = H; a.Dh = Dh; a.n_keys = n; a.causal = 0; a.scale = 1.f; a.bias = M->enc_bias;
             a.bias_len = 2 * E - 1; a.bias_zero = E - 1; a.q_pos0 = r0; a.out = M->attn; a.ldo = di;
-            a.partial = M->attn_partial; a.tickets = M->attn_tickets;
             CSD_TRY(attention(M, a, st));
             float* xr = M->xenc + (size_t)r0 * d;
             CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, xr, d, EPI_ADD, st));
@@ -494,19 +488,14 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
             if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = cnt_d; }
             CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         }
-        {
-            ProfScope ps(M, 2, st);
-            PdlLaunch L(dim3(m, H), dim3(64), 0, st);
-            CSD_CUDA(cudaLaunchKernelEx(&L.cfg, rope_append_kernel, M->qkv, 3 * di, 0, di, 2 * di, Dh, kv_len, c.max_seq,
-                                        (const float*)(c.arch == 0 ? M->rope_c : nullptr),
-                                        (const float*)(c.arch == 0 ? M->rope_s : nullptr), Kl, Vl));
-            count_launch();
-        }
         AttnArgs a;
         a.q = M->qkv; a.ldq = 3 * di; a.m = m; a.Kc = Kl; a.Vc = Vl; a.cap = c.max_seq; a.H = H; a.Dh = Dh;
         a.n_keys = kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
         if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = kv_len; }
-        a.out = M->attn; a.ldo = di; a.partial = M->attn_partial; a.tickets = M->attn_tickets;
+        a.out = M->attn; a.ldo = di;
+        // the block's own k and v rows go into the cache inside the attention kernel
+        a.k_new = M->qkv + di; a.v_new = M->qkv + 2 * di; a.ld_new = 3 * di;
+        if (c.arch == 0) { a.rope_cos = M->rope_c; a.rope_sin = M->rope_s; }
         if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
         CSD_TRY(attention(M, a, st));
         // output projection into the residual rows; hands them on to the norm that follows
@@ -523,8 +512,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
             AttnArgs x;
             x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
             x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
-            x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di; x.partial = M->attn_partial;
-            x.tickets = M->attn_tickets;
+            x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di;
             if (tc_o) { x.out_xs = M->xs_attn; x.out_xs_ld = di; }
             CSD_TRY(attention(M, x, st));
             LinOpt xo;

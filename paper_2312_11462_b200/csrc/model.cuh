@@ -26,8 +26,8 @@ struct csd_model {
     size_t layer_kv = 0, layer_x = 0;
     float *x = nullptr, *qkv = nullptr, *attn = nullptr, *act = nullptr, *xenc = nullptr, *qkv_enc = nullptr;
     float *rope_c = nullptr, *rope_s = nullptr, *dec_bias = nullptr, *enc_bias = nullptr;
-    float *gemm_partial = nullptr, *attn_partial = nullptr;
-    unsigned *gemm_tickets = nullptr, *attn_tickets = nullptr;
+    float* gemm_partial = nullptr;
+    unsigned* gemm_tickets = nullptr;
     __nv_bfloat16* xs_tmp = nullptr;    // three-term bf16 split of a GEMM's input rows (tensor-core path)
     float* ssq_tmp = nullptr;           // pieces of the rows' sums of squares written with it
     // activations handed from kernel to kernel in three-term form (tensor-core path)
