@@ -41,7 +41,7 @@ struct AttnParams {
     __nv_bfloat16* Kc; __nv_bfloat16* Vc; const float* bias; float* out;
     __nv_bfloat16* out_xs; int out_xs_ld;
     int* status;
-    int ldq, ld_new, m, cap, H, n_keys, n_old, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
+    int ldq, ld_new, m, cap, H, n_keys, n_old, early_loads, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
 };
 
@@ -96,8 +96,6 @@ block_attention_kernel(const AttnParams p) {
     if (tid < 32) { row_m[tid] = -INFINITY; row_l[tid] = 0.f; row_a[tid] = 1.f; }
     __syncthreads();
 
-    pdl_wait();       // q, the block's k and v rows and every committed cache row come from earlier kernels
-    pdl_trigger();
 
     // committed rows of tile `it` (the rest of the tile, if any, are the block's own rows)
     auto old_rows = [&](int it) {
@@ -112,7 +110,17 @@ block_attention_kernel(const AttnParams p) {
         bulk_load(Ks + (size_t)st * TILE * DH, Kh + (size_t)t0 * DH, bytes, &full[st]);
         bulk_load(Vs + (size_t)st * TILE * DH, Vh + (size_t)t0 * DH, bytes, &full[st]);
     };
-    if (tid == 0)
+    // Committed rows were written by the attention kernel of an earlier forward; between that
+    // kernel and this one the stream holds at least one kernel that waits for its predecessor
+    // before it lets its successor start, so those rows are complete and may be requested before
+    // this kernel's own dependency wait.  q and the block's k and v rows come from the kernel
+    // right before this one.  The encoder's self-attention reads rows the previous kernel wrote:
+    // there the requests wait too.
+    if (tid == 0 && p.early_loads)
+        for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
+    pdl_wait();
+    pdl_trigger();
+    if (tid == 0 && !p.early_loads)
         for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
 
     // ---- the block's rows: q (rotated) into shared memory; k (rotated) and v rounded to bf16, kept
@@ -370,6 +378,7 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     ap.status = status_word_device();
     ap.ldq = a.ldq; ap.m = a.m; ap.cap = a.cap; ap.H = a.H; ap.n_keys = a.n_keys;
     ap.n_old = append ? a.n_keys - 1 : total;
+    ap.early_loads = a.kv_settled ? 1 : 0;
     ap.causal = a.causal; ap.bias_len = a.bias_len; ap.bias_zero = a.bias_zero; ap.q_pos0 = a.q_pos0;
     ap.ldo = a.ldo; ap.scale = a.scale; ap.out_xs = a.out_xs; ap.out_xs_ld = a.out_xs_ld;
     ap.nsplit = attn_splits(total, a.H);

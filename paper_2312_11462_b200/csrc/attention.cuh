@@ -29,6 +29,10 @@ struct AttnArgs {
     int ld_new = 0;
     const float* rope_cos = nullptr;
     const float* rope_sin = nullptr;
+    // true when every cache row this call reads (other than the block's own) was complete before
+    // the kernel right before this one on the stream began; the tile requests then go out before
+    // the dependency wait
+    bool kv_settled = false;
 };
 
 int attn_splits(int total_keys, int H);

@@ -495,6 +495,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         a.out = M->attn; a.ldo = di;
         // the block's own k and v rows go into the cache inside the attention kernel
         a.k_new = M->qkv + di; a.v_new = M->qkv + 2 * di; a.ld_new = 3 * di;
+        a.kv_settled = true;      // committed rows date from earlier forwards
         if (c.arch == 0) { a.rope_cos = M->rope_c; a.rope_sin = M->rope_s; }
         if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
         CSD_TRY(attention(M, a, st));
@@ -513,6 +514,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
             x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
             x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
             x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di;
+            x.kv_settled = true;  // written once by the encoder pass
             if (tc_o) { x.out_xs = M->xs_attn; x.out_xs_ld = di; }
             CSD_TRY(attention(M, x, st));
             LinOpt xo;
