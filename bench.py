@@ -309,6 +309,110 @@ def run_review_only(args):
                       "n_acc": int(n_acc[0]), "out": int(out[0])}), flush=True)
 
 
+def run_configs(args):
+    """`--configs a,b,..` measures the other workload configurations (tiny cascade, accept sweep, T5-shaped
+    horizontal cascade, long-cache review) and prints one JSON line each; the default bench line is configuration 3."""
+    import torch
+    import workloads
+    from paper_2312_11462_b200 import binding as b
+    peak, _ = measured_peaks()
+    which = set(args.configs.split(","))
+
+    def timed(fn, n):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        e0.record()
+        for i in range(n):
+            fn(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return 1e3 * e0.elapsed_time(e1) / n          # microseconds per call
+
+    if "tiny" in which:
+        ts, ds = workloads.SHAPES["tiny_target"], workloads.SHAPES["tiny_draft"]
+        tb, db = workloads.make_weights(ts, 0, "cuda"), workloads.make_weights(ds, 1, "cuda")
+        prompt = workloads.make_prompt(ts.vocab, 32, seed=0)
+        nxt = torch.from_numpy(workloads.bigram_table(prompt, ts.vocab, seed=0)).cuda()
+        casc = b.Cascade([b.Model(ts, tb), b.Model(ds, db)], K_MATRIX, MAX_BLOCK, nxt, 32)
+        for _ in range(3):
+            casc.csd_cascade_generate(prompt, prompt, 64)
+        t0 = time.time()
+        for _ in range(10):
+            toks, st = casc.csd_cascade_generate(prompt, prompt, 64)
+        dt = (time.time() - t0) / 10
+        print(json.dumps({"config": "1 tiny cascade (prompt 32, 64 new, greedy, k=4)", "tokens_per_s": 64 / dt,
+                          "target_forwards_per_token": st["forwards"][0] / 64, "ms_per_generation": 1e3 * dt}), flush=True)
+
+    if "accept" in which:
+        rows = 64
+        for V in (4096, 32000, 128256):
+            for k in (1, 2, 4, 8, 16):
+                for sigma in ((0.1, 0.5, 2.0) if (V, k) == (32000, 4) else (0.5,)):
+                    # two input sets, alternated, so that a call never finds its own logits in L2 when they fit
+                    sets = [workloads.accept_case(rows, k, V, sigma, seed=7 + j, device="cuda") for j in range(2)]
+                    ws = b.csd_spec_accept_workspace(rows, k, V, "cuda")
+                    outs = (torch.empty(rows, dtype=torch.int32, device="cuda"),
+                            torch.empty(rows, dtype=torch.int32, device="cuda"))
+
+                    def call(i):
+                        t, d, tok = sets[i & 1]
+                        b.csd_spec_accept(t, d, tok, 1.0, seed=11, step=i, workspace=ws, out=outs)
+                    for i in range(4):
+                        call(i)
+                    us = timed(call, 20)
+                    nbytes = 4.0 * V * (2 * k + 1) * rows
+                    print(json.dumps({"config": "2 accept sweep", "V": V, "k": k, "sigma": sigma, "rows": rows,
+                                      "us": us, "algorithmic_MB": nbytes / 1e6, "GBps": nbytes / us / 1e3,
+                                      "frac_of_8TBps": nbytes / us / 1e3 / 8000.0,
+                                      "frac_of_measured": nbytes / us / 1e3 / peak,
+                                      "mean_accepted": float(outs[0].float().mean())}), flush=True)
+                    del sets, ws
+
+    if "long" in which:
+        ts = workloads.SHAPES["llama7b_long"]
+        tb = workloads.make_weights(ts, seed=100, device="cuda")
+        target = b.Model(ts, tb)
+        S = 2048
+        prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, S + 17, seed=5)).cuda()
+        for p0 in range(0, S, 16):
+            target.csd_review_forward(prompt[p0:p0 + 16], p0)
+        wbytes = 2.0 * (sum(int(np.prod(sh)) for n, _, sh in workloads.blob_layout(ts)[0]
+                            if "norm" not in n and n != "embed"))
+        for m in (2, 5, 9, 17):
+            blk = prompt[S:S + m].contiguous()
+            logits = torch.empty(m, ts.vocab, device="cuda")
+            for _ in range(3):
+                target.csd_review_forward(blk, S, logits)
+            us = timed(lambda i: target.csd_review_forward(blk, S, logits), 20)
+            kv = 2.0 * 2 * ts.n_layers * ts.d_inner * (S + m)
+            print(json.dumps({"config": "5 long-cache review", "S": S, "m": m, "review_us": us,
+                              "GBps": (wbytes + kv) / us / 1e3, "frac_of_8TBps": (wbytes + kv) / us / 1e3 / 8000.0,
+                              "frac_of_measured": (wbytes + kv) / us / 1e3 / peak}), flush=True)
+        target.close()
+        del tb
+
+    if "t5" in which:
+        shapes = [workloads.SHAPES[n] for n in ("t5xxl", "t5base", "t5small")]
+        blobs = [workloads.make_weights(sh, seed=200 + i, device="cuda") for i, sh in enumerate(shapes)]
+        models = [b.Model(sh, w) for sh, w in zip(shapes, blobs)]
+        enc = workloads.make_prompt(shapes[0].vocab, 256, seed=9)
+        nxt = torch.from_numpy(workloads.bigram_table(enc, shapes[0].vocab, seed=3)).cuda()
+        K = [[2, 2, 0], [0, 1, 4], [0, 0, 4]]
+        casc = b.Cascade(models, K, 4, nxt, 256)
+        start = np.array([0], dtype=np.int32)
+        casc.csd_cascade_generate(enc, start, 128, temperature=1.0, seed=1)
+        t0 = time.time()
+        toks, st = casc.csd_cascade_generate(enc, start, 128, temperature=1.0, seed=2)
+        dt = time.time() - t0
+        blk = torch.zeros(5, dtype=torch.int32, device="cuda")
+        logits = torch.empty(5, shapes[0].vocab, device="cuda")
+        us = timed(lambda i: models[0].csd_review_forward(blk, 64, logits), 10)
+        print(json.dumps({"config": "4 T5-xxl-shaped horizontal cascade (encoder 256, 128 new, T=1)",
+                          "tokens_per_s": len(toks) / dt, "prefill_ms": st["prefill_ms"], "decode_ms": st["decode_ms"],
+                          "target_forwards_per_token": st["forwards"][0] / max(len(toks), 1),
+                          "target_review_us_m5": us, "reviews": st["reviews"], "accepted": st["accepted"]}), flush=True)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -318,8 +422,11 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--review-only", type=int, default=0, help="profiling aid: only N review forwards of the target")
     ap.add_argument("--layers", type=int, default=0, help="with --review-only: cut the target to L layers")
+    ap.add_argument("--configs", default="", help="measure other configurations: tiny,accept,long,t5")
     args = ap.parse_args()
-    if args.review_only:
+    if args.configs:
+        run_configs(args)
+    elif args.review_only:
         run_review_only(args)
     elif args.impl == "reference":
         run_reference(args)

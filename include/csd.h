@@ -144,6 +144,11 @@ size_t csd_linear_workspace_bytes(int m, int N, int K);
  * weights, tcgen05.mma with fp32 accumulators in tensor memory) wherever it applies (K >= 64).
  * Both give the same result up to fp32 summation order; the switch exists to measure them. */
 csd_status csd_set_gemm_path(int path);
+/* Which kernel the block attention uses, process-wide: 0 = automatic (tensor cores, mma.sync on
+ * TMA-staged K/V tiles, for head dimensions 64 and 128; the CUDA-core kernel for 32), 1 = always
+ * the CUDA-core kernel.  Same result up to fp32 summation order and the 2^-17 relative error of the
+ * two-term bf16 form in which q and the softmax weights enter the MMAs. */
+csd_status csd_set_attention_path(int path);
 csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, int m, float* Y_dev,
                       void* workspace_dev, size_t workspace_bytes, void* stream);
 

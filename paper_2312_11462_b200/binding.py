@@ -79,6 +79,7 @@ lib.csd_review_forward.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
 lib.csd_model_profile.argtypes = [_vp, _i]
 lib.csd_model_profile_read.argtypes = [_vp, _vp, _vp]
 lib.csd_set_gemm_path.argtypes = [_i]
+lib.csd_set_attention_path.argtypes = [_i]
 lib.csd_linear_workspace_bytes.restype = _sz
 lib.csd_linear_workspace_bytes.argtypes = [_i, _i, _i]
 lib.csd_linear.argtypes = [_vp, _i, _i, _vp, _i, _vp, _vp, _sz, _vp]
@@ -202,6 +203,10 @@ def csd_linear(W: torch.Tensor, X: torch.Tensor, workspace: Optional[torch.Tenso
 
 def csd_set_gemm_path(path: int) -> None:
     _check("csd_set_gemm_path", lib.csd_set_gemm_path(path))
+
+
+def csd_set_attention_path(path: int) -> None:
+    _check("csd_set_attention_path", lib.csd_set_attention_path(path))
 
 
 def csd_linear_workspace(m: int, N: int, K: int, device) -> torch.Tensor:

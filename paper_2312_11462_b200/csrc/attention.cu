@@ -326,9 +326,356 @@ block_attention_kernel(const AttnParams p) {
     cluster.sync();       // no CTA leaves while another may still read its record
 }
 
+// -------------------------------------------------------------------------------------------------
+// Tensor-core variant (head dimension 64 or 128): the same walk over 64-key tiles, with the two
+// contractions of a tile on mma.sync (m16n8k16, bf16 operands, fp32 accumulators).  K and V tiles
+// arrive by tensor-map TMA copies with the 128-byte swizzle, which makes the ldmatrix reads of
+// their rows conflict-free; q and the softmax weights, fp32 quantities, enter the MMAs as a
+// bf16 pair (value = hi + lo, two MMAs), so the products keep 16 mantissa bits while K and V,
+// bf16 in the cache, are exact.  Warp w owns keys 8w..8w+7 of the tile in q.K^T and output
+// dimensions 16w..16w+15 in P.V; rows 16..31 (a 17-row block) are a second m16 tile.
+// -------------------------------------------------------------------------------------------------
+__device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void ldsm_x4_t(uint32_t addr, uint32_t (&r)[4]) {
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+__device__ __forceinline__ void mma_bf16(float (&d)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+// value = hi + lo with hi = bf16(value), lo = bf16(value - hi)
+__device__ __forceinline__ void split2(float v, __nv_bfloat16& hi, __nv_bfloat16& lo) {
+    hi = __float2bfloat16_rn(v);
+    lo = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
+
+template <int DH> struct MmaCfg {
+    static constexpr int QP = DH * 2 + 16;                   // bytes per q row: bf16 plus one 16-byte skew
+    static constexpr int PP = TILE * 2 + 16;                 // bytes per row of softmax weights
+    static constexpr int SP = TILE + 4;                      // floats per score row
+    static constexpr int REC = DH + 2;
+    static constexpr int NBOX = DH / 64;                     // 64-dimension (128-byte) boxes per row
+    static constexpr size_t TILE_BYTES = (size_t)TILE * DH * 2;
+    static constexpr size_t smem(int rows) {                 // rows = 16 or 32 operand rows
+        return 1024 + 2 * STAGES * TILE_BYTES + 2 * (size_t)rows * QP + (size_t)rows * SP * 4 + 2 * (size_t)rows * PP +
+               2 * (size_t)MAXM * DH * 2 + 3 * 32 * 4 + 64;
+    }
+};
+// byte offset of 16-byte chunk c (8 dimensions) of key row j inside a swizzled tile
+template <int DH> __device__ __forceinline__ uint32_t kv_off(int j, int c) {
+    return (uint32_t)((c >> 3) * (TILE * 128) + j * 128 + (((c & 7) ^ (j & 7)) << 4));
+}
+
+template <int DH, int MT>
+__global__ void __launch_bounds__(AT)
+block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid_constant__ CUtensorMap tmV,
+                           const AttnParams p) {
+    using C = MmaCfg<DH>;
+    constexpr int R = MT * 16;
+    extern __shared__ unsigned char smem_dyn[];
+    unsigned char* base = (unsigned char*)(((uintptr_t)smem_dyn + 1023) & ~(uintptr_t)1023);
+    unsigned char* Ks = base;                                        // [STAGES][tile], swizzled
+    unsigned char* Vs = Ks + STAGES * C::TILE_BYTES;
+    unsigned char* qh = Vs + STAGES * C::TILE_BYTES;                 // [R][QP] high parts of q; later the merge record
+    unsigned char* ql = qh + R * C::QP;
+    float* sc = reinterpret_cast<float*>(ql + R * C::QP);            // [R][SP]
+    unsigned char* ph = reinterpret_cast<unsigned char*>(sc + R * C::SP);   // [R][PP]
+    unsigned char* pl = ph + R * C::PP;
+    __nv_bfloat16* newK = reinterpret_cast<__nv_bfloat16*>(pl + R * C::PP); // [MAXM][DH]
+    __nv_bfloat16* newV = newK + MAXM * DH;
+    float* row_m = reinterpret_cast<float*>(newV + MAXM * DH);
+    float* row_l = row_m + 32;
+    float* row_a = row_l + 32;
+    uint64_t* full = reinterpret_cast<uint64_t*>(row_a + 32);
+
+    cg::cluster_group cluster = cg::this_cluster();
+    const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+    const int h = blockIdx.x, split = blockIdx.y;
+    const int m = p.m, half = DH / 2;
+    const int total = p.causal ? p.n_keys + m - 1 : p.n_keys;
+    const int s_begin = split * p.split_len;
+    const int s_end = min(total, s_begin + p.split_len);
+    const int n_tiles = s_end > s_begin ? (s_end - s_begin + TILE - 1) / TILE : 0;
+    __nv_bfloat16* Kh = p.Kc + (size_t)h * p.cap * DH;
+    __nv_bfloat16* Vh = p.Vc + (size_t)h * p.cap * DH;
+    const float* bias_h = p.bias ? p.bias + (size_t)h * p.bias_len : nullptr;
+
+    if (tid == 0) {
+        for (int s = 0; s < STAGES; ++s) mbar_init(&full[s], 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (tid < 32) { row_m[tid] = -INFINITY; row_l[tid] = 0.f; row_a[tid] = 1.f; }
+    // operand rows past the block stay zero (q, and the softmax weights, which are rewritten per tile only for real rows)
+    for (int i = tid; i < (2 * R * C::QP + R * C::SP * 4 + 2 * R * C::PP) / 16; i += AT)
+        reinterpret_cast<uint4*>(qh)[i] = make_uint4(0, 0, 0, 0);
+    __syncthreads();
+
+    auto request = [&](int it) {       // whole 64-row boxes: rows the block itself supplies are laid over afterwards
+        const int st = it % STAGES, row0 = h * p.cap + s_begin + it * TILE;
+        mbar_expect_tx(&full[st], 2 * (uint32_t)C::TILE_BYTES);
+#pragma unroll
+        for (int b = 0; b < C::NBOX; ++b) {
+            tma_load_2d(Ks + st * C::TILE_BYTES + b * (TILE * 128), &tmK, &full[st], b * 64, row0);
+            tma_load_2d(Vs + st * C::TILE_BYTES + b * (TILE * 128), &tmV, &full[st], b * 64, row0);
+        }
+    };
+    // (see the CUDA-core kernel above for why the requests may precede the dependency wait)
+    if (tid == 0 && p.early_loads)
+        for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
+    pdl_wait();
+    pdl_trigger();
+    if (tid == 0 && !p.early_loads)
+        for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
+
+    // ---- the block's rows: q rotated and split into its bf16 pair; k rotated, v, both rounded to bf16
+    for (int i = tid; i < m * half; i += AT) {
+        const int r = i / half, d = i % half, pos = p.n_old + r;
+        float c = 1.f, s = 0.f;
+        if (p.rope_cos) { c = p.rope_cos[(size_t)pos * half + d]; s = p.rope_sin[(size_t)pos * half + d]; }
+        const float* qr = p.q + (size_t)r * p.ldq + h * DH;
+        const float q0 = qr[d], q1 = qr[d + half];
+        __nv_bfloat16 h0, l0, h1, l1;
+        split2(q0 * c - q1 * s, h0, l0);
+        split2(q0 * s + q1 * c, h1, l1);
+        __nv_bfloat16* qhr = reinterpret_cast<__nv_bfloat16*>(qh + r * C::QP);
+        __nv_bfloat16* qlr = reinterpret_cast<__nv_bfloat16*>(ql + r * C::QP);
+        qhr[d] = h0; qhr[d + half] = h1; qlr[d] = l0; qlr[d + half] = l1;
+        if (p.k_new) {
+            const float* kr = p.k_new + (size_t)r * p.ld_new + h * DH;
+            const float* vr = p.v_new + (size_t)r * p.ld_new + h * DH;
+            const float k0 = kr[d], k1 = kr[d + half];
+            const __nv_bfloat16 ka = __float2bfloat16_rn(k0 * c - k1 * s), kb = __float2bfloat16_rn(k0 * s + k1 * c);
+            const __nv_bfloat16 va = __float2bfloat16_rn(vr[d]), vb = __float2bfloat16_rn(vr[d + half]);
+            newK[r * DH + d] = ka; newK[r * DH + d + half] = kb;
+            newV[r * DH + d] = va; newV[r * DH + d + half] = vb;
+            if (pos >= s_begin && pos < s_end) {
+                Kh[(size_t)pos * DH + d] = ka; Kh[(size_t)pos * DH + d + half] = kb;
+                Vh[(size_t)pos * DH + d] = va; Vh[(size_t)pos * DH + d + half] = vb;
+            }
+        }
+    }
+
+    float o[MT][2][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int t = 0; t < 2; ++t)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) o[mt][t][e] = 0.f;
+    const int lrow = lane & 7, lmat = lane >> 3;          // ldmatrix: this lane addresses row lrow of matrix lmat
+    const uint32_t qh_s = smem_u32(qh), ql_s = smem_u32(ql), ph_s = smem_u32(ph), pl_s = smem_u32(pl);
+
+    bool failed = false;
+    for (int it = 0; it < n_tiles; ++it) {
+        const int st = it % STAGES, t0 = s_begin + it * TILE;
+        const int ok = mbar_wait(&full[st], (uint32_t)(it / STAGES) & 1u);
+        if (__syncthreads_or(!ok)) {
+            if (!ok) mbar_wait(&full[st], (uint32_t)(it / STAGES) & 1u);
+            failed = true;
+            break;
+        }
+        unsigned char* Kt = Ks + st * C::TILE_BYTES;
+        unsigned char* Vt = Vs + st * C::TILE_BYTES;
+        const int valid = min(TILE, s_end - t0);
+        {
+            const int new_lo = max(t0, p.n_old), n_new = t0 + valid - new_lo;
+            for (int idx = tid; idx < n_new * (DH / 8); idx += AT) {
+                const int row = idx / (DH / 8), c = idx % (DH / 8), j = new_lo + row - t0, r = new_lo + row - p.n_old;
+                *reinterpret_cast<uint4*>(Kt + kv_off<DH>(j, c)) = *reinterpret_cast<const uint4*>(newK + r * DH + c * 8);
+                *reinterpret_cast<uint4*>(Vt + kv_off<DH>(j, c)) = *reinterpret_cast<const uint4*>(newV + r * DH + c * 8);
+            }
+            for (int idx = tid; idx < (TILE - valid) * (DH / 8); idx += AT) {
+                const int j = valid + idx / (DH / 8), c = idx % (DH / 8);
+                *reinterpret_cast<uint4*>(Vt + kv_off<DH>(j, c)) = make_uint4(0, 0, 0, 0);
+            }
+        }
+        __syncthreads();
+        // ---- scores of keys 8*warp .. 8*warp+7 for all rows
+        {
+            float sacc[MT][4];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) sacc[mt][e] = 0.f;
+            const uint32_t Kt_s = smem_u32(Kt);
+#pragma unroll
+            for (int ks2 = 0; ks2 < DH / 32; ++ks2) {
+                uint32_t kb[4];
+                ldsm_x4(Kt_s + kv_off<DH>(8 * warp + lrow, 4 * ks2 + lmat), kb);
+#pragma unroll
+                for (int hf = 0; hf < 2; ++hf) {
+                    const int ks = 2 * ks2 + hf;
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const uint32_t aoff = (uint32_t)((mt * 16 + (lmat & 1) * 8 + lrow) * C::QP + (2 * ks + (lmat >> 1)) * 16);
+                        uint32_t a[4];
+                        ldsm_x4(qh_s + aoff, a);
+                        mma_bf16(sacc[mt], a, kb[2 * hf], kb[2 * hf + 1]);
+                        ldsm_x4(ql_s + aoff, a);
+                        mma_bf16(sacc[mt], a, kb[2 * hf], kb[2 * hf + 1]);
+                    }
+                }
+            }
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const int r = mt * 16 + (lane >> 2) + (e >> 1) * 8, j = 8 * warp + (lane & 3) * 2 + (e & 1);
+                    if (r < m) {
+                        const int key = t0 + j, limit = p.causal ? p.n_keys + r : p.n_keys;
+                        float s = -INFINITY;
+                        if (key < s_end && key < limit) {
+                            s = sacc[mt][e] * p.scale;
+                            if (bias_h) {
+                                int bi = key - (p.q_pos0 + r) + p.bias_zero;
+                                bi = max(0, min(p.bias_len - 1, bi));
+                                s += bias_h[bi];
+                            }
+                        }
+                        sc[r * C::SP + j] = s;
+                    }
+                }
+        }
+        __syncthreads();
+        // ---- online softmax: warp w owns rows w, w+8, w+16; the weights leave as bf16 pairs
+        for (int r = warp; r < m; r += AT / 32) {
+            const float s0 = sc[r * C::SP + lane], s1 = sc[r * C::SP + lane + 32];
+            const float tmax = warp_max(fmaxf(s0, s1));
+            const float old = row_m[r];
+            const float nm = fmaxf(old, tmax);
+            float p0 = 0.f, p1 = 0.f, alpha = 1.f;
+            if (nm > -INFINITY) {
+                p0 = expf(s0 - nm);
+                p1 = expf(s1 - nm);
+                alpha = expf(old - nm);
+            }
+            __nv_bfloat16 h0, l0, h1, l1;
+            split2(p0, h0, l0);
+            split2(p1, h1, l1);
+            __nv_bfloat16* phr = reinterpret_cast<__nv_bfloat16*>(ph + r * C::PP);
+            __nv_bfloat16* plr = reinterpret_cast<__nv_bfloat16*>(pl + r * C::PP);
+            phr[lane] = h0; phr[lane + 32] = h1; plr[lane] = l0; plr[lane + 32] = l1;
+            // the sum runs over the weights as the MMA will see them
+            const float tsum = warp_sum((__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1)));
+            if (lane == 0) {
+                row_m[r] = nm;
+                row_l[r] = row_l[r] * alpha + tsum;
+                row_a[r] = alpha;
+            }
+        }
+        __syncthreads();
+        // ---- P.V for output dimensions 16*warp .. 16*warp+15
+        if (warp < DH / 16) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const float a0 = row_a[mt * 16 + (lane >> 2)], a1 = row_a[mt * 16 + (lane >> 2) + 8];
+#pragma unroll
+                for (int t = 0; t < 2; ++t) { o[mt][t][0] *= a0; o[mt][t][1] *= a0; o[mt][t][2] *= a1; o[mt][t][3] *= a1; }
+            }
+            const uint32_t Vt_s = smem_u32(Vt);
+#pragma unroll
+            for (int ks = 0; ks < TILE / 16; ++ks) {
+                uint32_t vb[4];
+                ldsm_x4_t(Vt_s + kv_off<DH>(16 * ks + (lmat & 1) * 8 + lrow, 2 * warp + (lmat >> 1)), vb);
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const uint32_t aoff = (uint32_t)((mt * 16 + (lmat & 1) * 8 + lrow) * C::PP + (2 * ks + (lmat >> 1)) * 16);
+                    uint32_t a[4];
+                    ldsm_x4(ph_s + aoff, a);
+                    mma_bf16(o[mt][0], a, vb[0], vb[1]);
+                    mma_bf16(o[mt][1], a, vb[2], vb[3]);
+                    ldsm_x4(pl_s + aoff, a);
+                    mma_bf16(o[mt][0], a, vb[0], vb[1]);
+                    mma_bf16(o[mt][1], a, vb[2], vb[3]);
+                }
+            }
+        }
+        __syncthreads();           // tile consumed: its stage may be filled again
+        if (tid == 0 && it + STAGES < n_tiles) {
+            fence_async_smem();
+            request(it + STAGES);
+        }
+    }
+    if (failed && tid == 0) set_status(p.status, CSD_ERR_TIMEOUT);
+
+
+    // element (mt, t, e) of `o`: row mt*16 + lane/4 (+8 for e >= 2), dimension 16*warp + 8*t + 2*(lane%4) + (e&1)
+    if (p.nsplit == 1) {
+        if (warp < DH / 16) {
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int hr = 0; hr < 2; ++hr) {
+                    const int r = mt * 16 + (lane >> 2) + hr * 8;
+                    if (r >= m) continue;
+                    const float inv = row_l[r] > 0.f ? 1.f / row_l[r] : 0.f;
+#pragma unroll
+                    for (int t = 0; t < 2; ++t) {
+                        const int d = 16 * warp + 8 * t + 2 * (lane & 3);
+                        float* dst = p.out + (size_t)r * p.ldo + h * DH + d;
+                        dst[0] = o[mt][t][2 * hr] * inv; dst[1] = o[mt][t][2 * hr + 1] * inv;
+                        if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, m, r, h * DH + d, dst[0], dst[1]);
+                    }
+                }
+        }
+        return;
+    }
+    float* rec = reinterpret_cast<float*>(qh);      // q is not needed any more (all threads are past the last tile)
+    if (warp < DH / 16) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int hr = 0; hr < 2; ++hr) {
+                const int r = mt * 16 + (lane >> 2) + hr * 8;
+                if (r >= m) continue;
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                    const int d = 16 * warp + 8 * t + 2 * (lane & 3);
+                    rec[r * C::REC + d] = o[mt][t][2 * hr];
+                    rec[r * C::REC + d + 1] = o[mt][t][2 * hr + 1];
+                }
+            }
+    }
+    if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
+    cluster.sync();
+    for (int i = split * AT + tid; i < m * DH; i += p.nsplit * AT) {
+        const int r = i / DH, d = i % DH;
+        float M = -INFINITY;
+        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(rec, s)[r * C::REC + DH]);
+        float num = 0.f, den = 0.f;
+        for (int s = 0; s < p.nsplit; ++s) {
+            const float* rs = cluster.map_shared_rank(rec, s) + r * C::REC;
+            const float ms = rs[DH];
+            if (ms > -INFINITY) {
+                const float w = expf(ms - M);
+                num = fmaf(rs[d], w, num);
+                den = fmaf(rs[DH + 1], w, den);
+            }
+        }
+        const float ov = den > 0.f ? num / den : 0.f;
+        p.out[(size_t)r * p.ldo + h * DH + d] = ov;
+        if (p.out_xs) {
+            uint16_t b1, b2, b3;
+            split3(ov, b1, b2, b3);
+            uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
+            xs[(size_t)r * p.out_xs_ld] = b1;
+            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
+            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
+        }
+    }
+    cluster.sync();       // no CTA leaves while another may still read its record
+}
 // One 64-key tile per CTA while that keeps the splits of a head inside one portable cluster (8)
 // and the grid near two CTAs per SM: short caches are latency-bound, and more splits mean more
 // tiles in flight at once; long caches walk several tiles per CTA, two requests ahead.
+static bool g_attn_cuda_cores = false;
+void set_attention_cuda_cores(bool on) { g_attn_cuda_cores = on; }
+
 int attn_splits(int total_keys, int H) {
     int by_sm = (2 * 148 + H - 1) / H;
     int by_len = (total_keys + TILE - 1) / TILE;
@@ -336,6 +683,21 @@ int attn_splits(int total_keys, int H) {
     if (n < 1) n = 1;
     if (n > MAX_SPLITS) n = MAX_SPLITS;
     return n;
+}
+
+static void attn_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, const AttnParams& ap, size_t smem,
+                               cudaStream_t st) {
+    cfg = cudaLaunchConfig_t{};
+    cfg.gridDim = dim3((unsigned)ap.H, (unsigned)ap.nsplit);
+    cfg.blockDim = dim3(AT);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    attr[1].id = cudaLaunchAttributeClusterDimension;      // the splits of one head exchange results on chip
+    attr[1].val.clusterDim.x = 1; attr[1].val.clusterDim.y = (unsigned)ap.nsplit; attr[1].val.clusterDim.z = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
 }
 
 template <int DH>
@@ -346,19 +708,27 @@ static csd_status launch_dh(const AttnParams& ap, cudaStream_t st) {
         CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)AttnCfg<DH>::SMEM));
         attr_set = true;
     }
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3((unsigned)ap.H, (unsigned)ap.nsplit);
-    cfg.blockDim = dim3(AT);
-    cfg.dynamicSmemBytes = AttnCfg<DH>::SMEM;
-    cfg.stream = st;
+    cudaLaunchConfig_t cfg;
     cudaLaunchAttribute attr[2];
-    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
-    attr[0].val.programmaticStreamSerializationAllowed = 1;
-    attr[1].id = cudaLaunchAttributeClusterDimension;      // the splits of one head exchange results on chip
-    attr[1].val.clusterDim.x = 1; attr[1].val.clusterDim.y = (unsigned)ap.nsplit; attr[1].val.clusterDim.z = 1;
-    cfg.attrs = attr;
-    cfg.numAttrs = 2;
+    attn_launch_config(cfg, attr, ap, AttnCfg<DH>::SMEM, st);
     CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, ap));
+    count_launch();
+    return CSD_OK;
+}
+
+template <int DH, int MT>
+static csd_status launch_mma(const CUtensorMap& tk, const CUtensorMap& tv, const AttnParams& ap, cudaStream_t st) {
+    auto kern = block_attention_mma_kernel<DH, MT>;
+    static bool attr_set = false;
+    const size_t smem = MmaCfg<DH>::smem(MT * 16);
+    if (!attr_set) {
+        CSD_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        attr_set = true;
+    }
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[2];
+    attn_launch_config(cfg, attr, ap, smem, st);
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, tk, tv, ap));
     count_launch();
     return CSD_OK;
 }
@@ -385,6 +755,14 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;
     ap.nsplit = (total + ap.split_len - 1) / ap.split_len;
+    // head dimensions 64 and 128 run on the tensor cores; the caches then need tensor maps (rows = all heads' positions)
+    if ((a.Dh == 64 || a.Dh == 128) && !g_attn_cuda_cores) {
+        CUtensorMap tk, tv;
+        if (tensor_map_2d(a.Kc, a.H * a.cap, a.Dh, TILE, &tk) && tensor_map_2d(a.Vc, a.H * a.cap, a.Dh, TILE, &tv)) {
+            if (a.Dh == 64) return a.m <= 16 ? launch_mma<64, 1>(tk, tv, ap, st) : launch_mma<64, 2>(tk, tv, ap, st);
+            return a.m <= 16 ? launch_mma<128, 1>(tk, tv, ap, st) : launch_mma<128, 2>(tk, tv, ap, st);
+        }
+    }
     switch (a.Dh) {
         case 32: return launch_dh<32>(ap, st);
         case 64: return launch_dh<64>(ap, st);
@@ -394,3 +772,9 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
 }
 
 }  // namespace csd
+
+extern "C" csd_status csd_set_attention_path(int path) {
+    if (path < 0 || path > 1) return CSD_ERR_INVALID_ARG;
+    csd::set_attention_cuda_cores(path == 1);
+    return CSD_OK;
+}

@@ -36,6 +36,7 @@ struct AttnArgs {
 };
 
 int attn_splits(int total_keys, int H);
+void set_attention_cuda_cores(bool on);   // true: always the CUDA-core kernel (for comparison runs)
 csd_status launch_attention(const AttnArgs& a, cudaStream_t st);
 
 }  // namespace csd

@@ -13,12 +13,15 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module", params=[1, 2], ids=["cuda-core", "tensor-core"])
 def b(request):
-    """Every test here runs once per GEMM kernel: 128-bit loads + fp32 FMA, and TMA + tcgen05."""
+    """Every test here runs once per kernel family: CUDA-core GEMM (128-bit loads + fp32 FMA) with the
+    CUDA-core attention, and tensor-core GEMM (TMA + tcgen05) with the tensor-core attention."""
     require_gpu()
     from paper_2312_11462_b200 import binding
     binding.csd_set_gemm_path(request.param)
+    binding.csd_set_attention_path(1 if request.param == 1 else 0)
     yield binding
     binding.csd_set_gemm_path(0)
+    binding.csd_set_attention_path(0)
 
 
 def check(got, ref, what):

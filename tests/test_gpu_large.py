@@ -58,6 +58,7 @@ def test_7b_width_shallow_stack(b, orc, path):
     blob = workloads.make_weights(shape, seed=100, device="cuda")
     seq = workloads.make_prompt(shape.vocab, 24, seed=1000)
     b.csd_set_gemm_path(path)
+    b.csd_set_attention_path(1 if path == 1 else 0)
     try:
         gm, om = b.Model(shape, blob), orc.Model(shape, orc.blob_to_u16(blob))
         for pos, m in ((0, 17), (17, 5), (22, 1)):
@@ -69,9 +70,19 @@ def test_7b_width_shallow_stack(b, orc, path):
         assert b.csd_device_status() == 0
     finally:
         b.csd_set_gemm_path(0)
+        b.csd_set_attention_path(0)
 
 
-def test_long_cache_review_blocks(b, orc):
+@pytest.mark.parametrize("attn_path", [0, 1], ids=["tensor-core-attention", "cuda-core-attention"])
+def test_long_cache_review_blocks(b, orc, attn_path):
+    b.csd_set_attention_path(attn_path)
+    try:
+        long_cache_review_blocks(b, orc)
+    finally:
+        b.csd_set_attention_path(0)
+
+
+def long_cache_review_blocks(b, orc):
     shape = llama_shape(2, 1024, 8, 2752, 8000, 2624)
     blob = workloads.make_weights(shape, seed=21, device="cuda")
     toks = workloads.make_prompt(shape.vocab, 2100, seed=3)
