@@ -61,6 +61,48 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* xs, int ld, int m, in
     base[((size_t)(2 * m + r) * ld) >> 1] = a3 | ((uint32_t)c3 << 16);
 }
 
+
+// Merge of the splits' records (unnormalised output row, running max, running sum) through
+// distributed shared memory: the CTAs of a head share out the m*DH output elements; each thread
+// first fetches everything it needs from all splits in one batch of independent remote loads.
+template <int DH, int REC>
+__device__ __forceinline__ void merge_splits(cg::cluster_group& cluster, float* rec, const AttnParams& p, int h, int split) {
+    const int m = p.m;
+    for (int i = split * AT + threadIdx.x; i < m * DH; i += p.nsplit * AT) {
+        const int r = i / DH, d = i % DH;
+        float ms[MAX_SPLITS], ls[MAX_SPLITS], vs[MAX_SPLITS];
+#pragma unroll
+        for (int s = 0; s < MAX_SPLITS; ++s) {
+            ms[s] = -INFINITY; ls[s] = 0.f; vs[s] = 0.f;
+            if (s < p.nsplit) {
+                const float* rs = cluster.map_shared_rank(rec, s) + r * REC;
+                ms[s] = rs[DH]; ls[s] = rs[DH + 1]; vs[s] = rs[d];
+            }
+        }
+        float M = -INFINITY;
+#pragma unroll
+        for (int s = 0; s < MAX_SPLITS; ++s) M = fmaxf(M, ms[s]);
+        float num = 0.f, den = 0.f;
+#pragma unroll
+        for (int s = 0; s < MAX_SPLITS; ++s)
+            if (ms[s] > -INFINITY) {
+                const float w = expf(ms[s] - M);
+                num = fmaf(vs[s], w, num);
+                den = fmaf(ls[s], w, den);
+            }
+        const float ov = den > 0.f ? num / den : 0.f;
+        p.out[(size_t)r * p.ldo + h * DH + d] = ov;
+        if (p.out_xs) {
+            uint16_t b1, b2, b3;
+            split3(ov, b1, b2, b3);
+            uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
+            xs[(size_t)r * p.out_xs_ld] = b1;
+            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
+            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
+        }
+    }
+}
+
 template <int DH>
 __global__ void __launch_bounds__(AT)
 block_attention_kernel(const AttnParams p) {
@@ -298,31 +340,7 @@ block_attention_kernel(const AttnParams p) {
     }
     if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
     cluster.sync();
-    for (int i = split * AT + tid; i < m * DH; i += p.nsplit * AT) {
-        const int r = i / DH, d = i % DH;
-        float M = -INFINITY;
-        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(rec, s)[r * C::REC + DH]);
-        float num = 0.f, den = 0.f;
-        for (int s = 0; s < p.nsplit; ++s) {
-            const float* rs = cluster.map_shared_rank(rec, s) + r * C::REC;
-            const float ms = rs[DH];
-            if (ms > -INFINITY) {
-                const float w = expf(ms - M);
-                num = fmaf(rs[d], w, num);
-                den = fmaf(rs[DH + 1], w, den);
-            }
-        }
-        const float o = den > 0.f ? num / den : 0.f;
-        p.out[(size_t)r * p.ldo + h * DH + d] = o;
-        if (p.out_xs) {
-            uint16_t b1, b2, b3;
-            split3(o, b1, b2, b3);
-            uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
-            xs[(size_t)r * p.out_xs_ld] = b1;
-            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
-            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
-        }
-    }
+    merge_splits<DH, C::REC>(cluster, rec, p, h, split);
     cluster.sync();       // no CTA leaves while another may still read its record
 }
 
@@ -427,35 +445,65 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     // (see the CUDA-core kernel above for why the requests may precede the dependency wait)
     if (tid == 0 && p.early_loads)
         for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
+    // this thread's (row, dimension pair) items of the block; their rotation factors are constants
+    constexpr int ITEMS = (MAXM * (DH / 2) + AT - 1) / AT;
+    float rc[ITEMS], rs[ITEMS];
+#pragma unroll
+    for (int e = 0; e < ITEMS; ++e) {
+        const int i = tid + e * AT;
+        rc[e] = 1.f; rs[e] = 0.f;
+        if (i < m * half && p.rope_cos) {
+            const size_t at = (size_t)(p.n_old + i / half) * half + i % half;
+            rc[e] = p.rope_cos[at]; rs[e] = p.rope_sin[at];
+        }
+    }
     pdl_wait();
     pdl_trigger();
     if (tid == 0 && !p.early_loads)
         for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
 
-    // ---- the block's rows: q rotated and split into its bf16 pair; k rotated, v, both rounded to bf16
-    for (int i = tid; i < m * half; i += AT) {
-        const int r = i / half, d = i % half, pos = p.n_old + r;
-        float c = 1.f, s = 0.f;
-        if (p.rope_cos) { c = p.rope_cos[(size_t)pos * half + d]; s = p.rope_sin[(size_t)pos * half + d]; }
-        const float* qr = p.q + (size_t)r * p.ldq + h * DH;
-        const float q0 = qr[d], q1 = qr[d + half];
-        __nv_bfloat16 h0, l0, h1, l1;
-        split2(q0 * c - q1 * s, h0, l0);
-        split2(q0 * s + q1 * c, h1, l1);
-        __nv_bfloat16* qhr = reinterpret_cast<__nv_bfloat16*>(qh + r * C::QP);
-        __nv_bfloat16* qlr = reinterpret_cast<__nv_bfloat16*>(ql + r * C::QP);
-        qhr[d] = h0; qhr[d + half] = h1; qlr[d] = l0; qlr[d + half] = l1;
-        if (p.k_new) {
-            const float* kr = p.k_new + (size_t)r * p.ld_new + h * DH;
-            const float* vr = p.v_new + (size_t)r * p.ld_new + h * DH;
-            const float k0 = kr[d], k1 = kr[d + half];
-            const __nv_bfloat16 ka = __float2bfloat16_rn(k0 * c - k1 * s), kb = __float2bfloat16_rn(k0 * s + k1 * c);
-            const __nv_bfloat16 va = __float2bfloat16_rn(vr[d]), vb = __float2bfloat16_rn(vr[d + half]);
-            newK[r * DH + d] = ka; newK[r * DH + d + half] = kb;
-            newV[r * DH + d] = va; newV[r * DH + d + half] = vb;
-            if (pos >= s_begin && pos < s_end) {
-                Kh[(size_t)pos * DH + d] = ka; Kh[(size_t)pos * DH + d + half] = kb;
-                Vh[(size_t)pos * DH + d] = va; Vh[(size_t)pos * DH + d + half] = vb;
+    // ---- the block's rows: q rotated and split into its bf16 pair; k rotated, v, both rounded to bf16.
+    //      All loads first (one round trip), then the arithmetic and the stores.
+    {
+        float qv[ITEMS][2], kv[ITEMS][2], vv[ITEMS][2];
+#pragma unroll
+        for (int e = 0; e < ITEMS; ++e) {
+            const int i = tid + e * AT;
+            if (i < m * half) {
+                const int r = i / half, d = i % half;
+                const float* qr = p.q + (size_t)r * p.ldq + h * DH;
+                qv[e][0] = qr[d]; qv[e][1] = qr[d + half];
+                if (p.k_new) {
+                    const float* kr = p.k_new + (size_t)r * p.ld_new + h * DH;
+                    const float* vr = p.v_new + (size_t)r * p.ld_new + h * DH;
+                    kv[e][0] = kr[d]; kv[e][1] = kr[d + half];
+                    vv[e][0] = vr[d]; vv[e][1] = vr[d + half];
+                }
+            }
+        }
+#pragma unroll
+        for (int e = 0; e < ITEMS; ++e) {
+            const int i = tid + e * AT;
+            if (i < m * half) {
+                const int r = i / half, d = i % half, pos = p.n_old + r;
+                const float c = rc[e], s = rs[e];
+                __nv_bfloat16 h0, l0, h1, l1;
+                split2(qv[e][0] * c - qv[e][1] * s, h0, l0);
+                split2(qv[e][0] * s + qv[e][1] * c, h1, l1);
+                __nv_bfloat16* qhr = reinterpret_cast<__nv_bfloat16*>(qh + r * C::QP);
+                __nv_bfloat16* qlr = reinterpret_cast<__nv_bfloat16*>(ql + r * C::QP);
+                qhr[d] = h0; qhr[d + half] = h1; qlr[d] = l0; qlr[d + half] = l1;
+                if (p.k_new) {
+                    const __nv_bfloat16 ka = __float2bfloat16_rn(kv[e][0] * c - kv[e][1] * s);
+                    const __nv_bfloat16 kb = __float2bfloat16_rn(kv[e][0] * s + kv[e][1] * c);
+                    const __nv_bfloat16 va = __float2bfloat16_rn(vv[e][0]), vb = __float2bfloat16_rn(vv[e][1]);
+                    newK[r * DH + d] = ka; newK[r * DH + d + half] = kb;
+                    newV[r * DH + d] = va; newV[r * DH + d + half] = vb;
+                    if (pos >= s_begin && pos < s_end) {
+                        Kh[(size_t)pos * DH + d] = ka; Kh[(size_t)pos * DH + d + half] = kb;
+                        Vh[(size_t)pos * DH + d] = va; Vh[(size_t)pos * DH + d + half] = vb;
+                    }
+                }
             }
         }
     }
@@ -643,31 +691,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     }
     if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
     cluster.sync();
-    for (int i = split * AT + tid; i < m * DH; i += p.nsplit * AT) {
-        const int r = i / DH, d = i % DH;
-        float M = -INFINITY;
-        for (int s = 0; s < p.nsplit; ++s) M = fmaxf(M, cluster.map_shared_rank(rec, s)[r * C::REC + DH]);
-        float num = 0.f, den = 0.f;
-        for (int s = 0; s < p.nsplit; ++s) {
-            const float* rs = cluster.map_shared_rank(rec, s) + r * C::REC;
-            const float ms = rs[DH];
-            if (ms > -INFINITY) {
-                const float w = expf(ms - M);
-                num = fmaf(rs[d], w, num);
-                den = fmaf(rs[DH + 1], w, den);
-            }
-        }
-        const float ov = den > 0.f ? num / den : 0.f;
-        p.out[(size_t)r * p.ldo + h * DH + d] = ov;
-        if (p.out_xs) {
-            uint16_t b1, b2, b3;
-            split3(ov, b1, b2, b3);
-            uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
-            xs[(size_t)r * p.out_xs_ld] = b1;
-            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
-            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
-        }
-    }
+    merge_splits<DH, C::REC>(cluster, rec, p, h, split);
     cluster.sync();       // no CTA leaves while another may still read its record
 }
 // One 64-key tile per CTA while that keeps the splits of a head inside one portable cluster (8)
