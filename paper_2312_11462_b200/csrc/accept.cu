@@ -1,12 +1,19 @@
 // Review rule of speculative sampling (Section 2; lenience / greedy: Section 3.1) as three
-// passes over the vocabulary:
-//   stats   one streaming pass over all (2k+1) logit vectors of every row: per-chunk max,
-//           arg-max and sum of exponentials (fp32).  This is the HBM-bound part.
-//   decide  per row: merge the chunk partials, run the accept tests left to right with the
-//           Philox uniforms, find the first rejection n.
-//   resample (temperature > 0 only) per row, at position n only: total mass of the residual
-//           max(0, p - q) (or of p after k acceptances) and the inverse-CDF pick, in fp64 so
-//           that the chosen token does not depend on the summation order.
+// kernels over the vocabulary:
+//   stats    one streaming pass over all (2k+1) logit vectors of every row: per 8192-logit piece
+//            the max, arg-max and sum of exponentials (fp32).  This is the HBM-bound part: a
+//            warp owns a piece, keeps 8 x 16 bytes per lane in flight with the next 8 already
+//            requested, and needs no block-wide synchronisation.
+//   decide   per row: merge the pieces, run the accept tests of all positions in parallel with
+//            the Philox uniforms, find the first rejection n.
+//   resample (temperature > 0 only) per row, at position n only, in fp64 so that the chosen token
+//            does not depend on summation order or on fp32 rounding: first the per-chunk sums
+//            of the exponentials (the normalisers), then per chunk the mass of the residual
+//            max(0, p - q) (or of p after k acceptances); the CTA that finishes a row last takes
+//            the inverse-CDF pick.  exp() here is a short fp64 routine of this file (argument
+//            reduction by ln 2 and a degree-11 Taylor polynomial, relative error below 1e-13 on
+//            the arguments that occur, x <= 0), and every division is a multiplication by a
+//            reciprocal formed once.
 #include "common.cuh"
 #include "philox.cuh"
 #include <mutex>
@@ -14,14 +21,15 @@
 namespace csd {
 
 constexpr int ST_THREADS = 256;
-constexpr int ST_CHUNK = 4096;   // logits per CTA of the stats pass
+constexpr int ST_CHUNK = 8192;   // logits per warp item of the stats pass
+constexpr int ST_SUB = 1024;     // logits a warp has in registers at a time (8 x float4 per lane)
 constexpr int RS_THREADS = 256;
 constexpr int RS_PER_THREAD = 8;
-constexpr int RS_CHUNK = RS_THREADS * RS_PER_THREAD;  // logits per CTA of the resample passes
+constexpr int RS_CHUNK = RS_THREADS * RS_PER_THREAD;  // logits per CTA of the resample pass
 
 struct __align__(16) StatPartial {
     float mx;
-    float sum;   // sum exp((x - mx) * invT) over the chunk
+    float sum;   // sum exp((x - mx) * invT) over the piece
     int arg;     // smallest index attaining mx
     int pad;
 };
@@ -39,73 +47,86 @@ struct __align__(16) RowInfo {
 };
 
 // ---------------------------------------------------------------------------------------------
-// stats pass
+// stats pass: grid-stride loop of warps over (vector, piece) items
 // ---------------------------------------------------------------------------------------------
 template <bool VEC>
-__global__ void __launch_bounds__(ST_THREADS)
-accept_stats_kernel(const float* __restrict__ tl, const float* __restrict__ dl, long long n_tvec, int V,
-                    float invT, int greedy, StatPartial* __restrict__ out, int nchunk) {
-    const long long vec = blockIdx.x;
-    const int chunk = blockIdx.y;
-    const float* src = vec < n_tvec ? tl + vec * (long long)V : dl + (vec - n_tvec) * (long long)V;
-    const int base = chunk * ST_CHUNK;
-    const int tid = threadIdx.x;
-    constexpr int PER = ST_CHUNK / ST_THREADS;  // 16
-    float v[PER];
+__device__ __forceinline__ void load_sub(const float* __restrict__ src, int e0, int V, int lane, float (&v)[32]) {
     if (VEC) {
 #pragma unroll
-        for (int j = 0; j < PER / 4; ++j) {
-            int e = base + 4 * (tid + ST_THREADS * j);
+        for (int j = 0; j < 8; ++j) {
+            const int e = e0 + 4 * (lane + 32 * j);
             float4 f = make_float4(-INFINITY, -INFINITY, -INFINITY, -INFINITY);
             if (e < V) f = __ldcs(reinterpret_cast<const float4*>(src + e));
             v[4 * j + 0] = f.x; v[4 * j + 1] = f.y; v[4 * j + 2] = f.z; v[4 * j + 3] = f.w;
         }
     } else {
 #pragma unroll
-        for (int j = 0; j < PER; ++j) {
-            int e = base + tid + ST_THREADS * j;
+        for (int j = 0; j < 32; ++j) {
+            const int e = e0 + lane + 32 * j;
             v[j] = e < V ? __ldcs(src + e) : -INFINITY;
         }
     }
-    // thread-local max with the smallest index attaining it
-    float mx = -INFINITY;
-    int arg = 0x7fffffff;
+}
+template <bool VEC> __device__ __forceinline__ int sub_index(int e0, int lane, int j) {
+    return VEC ? e0 + 4 * (lane + 32 * (j >> 2)) + (j & 3) : e0 + lane + 32 * j;
+}
+
+template <bool VEC>
+__global__ void __launch_bounds__(ST_THREADS, 2)
+accept_stats_kernel(const float* __restrict__ tl, const float* __restrict__ dl, long long n_tvec, int V,
+                    float invT, int greedy, StatPartial* __restrict__ out, int nchunk, long long items) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = (long long)gridDim.x * (ST_THREADS / 32);
+    for (long long item = (long long)blockIdx.x * (ST_THREADS / 32) + (threadIdx.x >> 5); item < items; item += warps) {
+        const long long vec = item / nchunk;
+        const int chunk = (int)(item % nchunk);
+        const float* src = vec < n_tvec ? tl + vec * (long long)V : dl + (vec - n_tvec) * (long long)V;
+        const int base = chunk * ST_CHUNK;
+        const int nsub = (min(V, base + ST_CHUNK) - base + ST_SUB - 1) / ST_SUB;
+        float mx = -INFINITY, sum = 0.f;
+        int arg = 0x7fffffff;
+        float cur[32], nxt[32];
+        load_sub<VEC>(src, base, V, lane, cur);
+        for (int s = 0; s < nsub; ++s) {
+            const int e0 = base + s * ST_SUB;
+            if (s + 1 < nsub) load_sub<VEC>(src, e0 + ST_SUB, V, lane, nxt);     // in flight while this batch is reduced
+            // batch max with the smallest index attaining it (indices grow with j inside a lane)
+            float bm = -INFINITY;
+            int ba = 0x7fffffff;
 #pragma unroll
-    for (int j = 0; j < PER; ++j) {
-        int e = VEC ? base + 4 * (tid + ST_THREADS * (j / 4)) + (j & 3) : base + tid + ST_THREADS * j;
-        if (v[j] > mx || (v[j] == mx && e < arg)) { mx = v[j]; arg = e; }
-    }
+            for (int j = 0; j < 32; ++j)
+                if (cur[j] > bm) { bm = cur[j]; ba = sub_index<VEC>(e0, lane, j); }
+            if (bm > mx) {          // later batches hold larger indices, so ">" keeps the earliest arg-max
+                sum = mx > -INFINITY ? sum * __expf((mx - bm) * invT) : 0.f;
+                mx = bm; arg = ba;
+            }
+            if (!greedy && mx > -INFINITY) {
+                float a = 0.f;
 #pragma unroll
-    for (int o = 16; o > 0; o >>= 1) {
-        float om = __shfl_xor_sync(0xffffffffu, mx, o);
-        int oa = __shfl_xor_sync(0xffffffffu, arg, o);
-        if (om > mx || (om == mx && oa < arg)) { mx = om; arg = oa; }
-    }
-    __shared__ float s_mx[ST_THREADS / 32];
-    __shared__ int s_arg[ST_THREADS / 32];
-    __shared__ float s_sum[ST_THREADS / 32];
-    const int warp = tid >> 5, lane = tid & 31;
-    if (lane == 0) { s_mx[warp] = mx; s_arg[warp] = arg; }
-    __syncthreads();
-    mx = s_mx[0]; arg = s_arg[0];
+                for (int j = 0; j < 32; ++j) a += __expf((cur[j] - mx) * invT);
+                sum += a;
+            }
+            if (s + 1 < nsub) {
 #pragma unroll
-    for (int w = 1; w < ST_THREADS / 32; ++w)
-        if (s_mx[w] > mx || (s_mx[w] == mx && s_arg[w] < arg)) { mx = s_mx[w]; arg = s_arg[w]; }
-    float sum = 0.f;
-    if (!greedy && mx > -INFINITY) {
+                for (int j = 0; j < 32; ++j) cur[j] = nxt[j];
+            }
+        }
+        // lanes -> warp
+        float wm = mx;
+        int wa = arg;
 #pragma unroll
-        for (int j = 0; j < PER; ++j) sum += __expf((v[j] - mx) * invT);
-    }
-    sum = warp_sum(sum);
-    if (lane == 0) s_sum[warp] = sum;
-    __syncthreads();
-    if (tid == 0) {
-        float tot = 0.f;
-#pragma unroll
-        for (int w = 0; w < ST_THREADS / 32; ++w) tot += s_sum[w];
-        StatPartial p;
-        p.mx = mx; p.sum = tot; p.arg = arg; p.pad = 0;
-        out[vec * nchunk + chunk] = p;
+        for (int o = 16; o > 0; o >>= 1) {
+            const float om = __shfl_xor_sync(0xffffffffu, wm, o);
+            const int oa = __shfl_xor_sync(0xffffffffu, wa, o);
+            if (om > wm || (om == wm && oa < wa)) { wm = om; wa = oa; }
+        }
+        float scaled = (!greedy && mx > -INFINITY) ? sum * __expf((mx - wm) * invT) : 0.f;
+        scaled = warp_sum(scaled);
+        if (lane == 0) {
+            StatPartial p;
+            p.mx = wm; p.sum = scaled; p.arg = wa; p.pad = 0;
+            out[item] = p;
+        }
     }
 }
 
@@ -118,34 +139,44 @@ __global__ void __launch_bounds__(128)
 accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl, const int* __restrict__ onehot,
                      const int* __restrict__ tokens, int rows, int k, int V, float temperature, float lenience,
                      uint64_t seed, uint64_t step, const StatPartial* __restrict__ part, int nchunk,
-                     int* __restrict__ n_acc, int* __restrict__ out_tok, RowInfo* __restrict__ info, int* status) {
+                     int* __restrict__ n_acc, int* __restrict__ out_tok, RowInfo* __restrict__ info,
+                     unsigned* __restrict__ tickets, int* status) {
     const int row = blockIdx.x;
     __shared__ float s_mx[2 * MAX_K + 1];
     __shared__ float s_z[2 * MAX_K + 1];
     __shared__ int s_arg[2 * MAX_K + 1];
+    __shared__ int s_acc[MAX_K], s_x[MAX_K], s_point[MAX_K];
+    __shared__ double s_u2[MAX_K];
     const bool greedy = temperature == 0.f;
     const float invT = greedy ? 1.f : 1.f / temperature;
     const int nvec_row = dl ? 2 * k + 1 : k + 1;
     const long long n_tvec = (long long)rows * (k + 1);
+    // ---- merge the pieces of every vector of this row (one thread per vector, one pass)
     for (int i = threadIdx.x; i < nvec_row; i += blockDim.x) {
-        long long vec = i <= k ? (long long)row * (k + 1) + i : n_tvec + (long long)row * k + (i - k - 1);
+        const long long vec = i <= k ? (long long)row * (k + 1) + i : n_tvec + (long long)row * k + (i - k - 1);
         const StatPartial* p = part + vec * nchunk;
-        float mx = p[0].mx;
-        int arg = p[0].arg;
-        for (int c = 1; c < nchunk; ++c)
-            if (p[c].mx > mx) { mx = p[c].mx; arg = p[c].arg; }
-        float z = 0.f;
-        if (!greedy)
-            for (int c = 0; c < nchunk; ++c)
-                if (p[c].mx > -INFINITY) z += p[c].sum * __expf((p[c].mx - mx) * invT);
-        s_mx[i] = mx; s_z[i] = z; s_arg[i] = arg;
+        float mx = -INFINITY, z = 0.f;
+        int arg = 0x7fffffff;
+#pragma unroll 4
+        for (int c = 0; c < nchunk; ++c) {
+            const StatPartial q = p[c];
+            if (q.mx > mx) {        // pieces come in index order, so ">" keeps the earliest arg-max
+                z = mx > -INFINITY ? z * __expf((mx - q.mx) * invT) : 0.f;
+                mx = q.mx; arg = q.arg;
+                z += q.sum;
+            } else if (q.mx > -INFINITY) {
+                z += q.sum * __expf((q.mx - mx) * invT);
+            }
+        }
+        s_mx[i] = mx; s_z[i] = greedy ? 0.f : z; s_arg[i] = arg;
     }
+    if (threadIdx.x == 0 && tickets) tickets[row] = 0u;     // for the resample pass that follows
     __syncthreads();
-    if (threadIdx.x != 0) return;
     const int* tok = tokens + (long long)row * k;
     RowInfo ri;
     ri.n = k; ri.mode = MODE_DONE; ri.x = 0; ri.pad = 0; ri.max_t = 0; ri.max_q = 0; ri.u2 = 0;
     if (greedy) {
+        if (threadIdx.x != 0) return;
         int n = 0;
         while (n < k && tok[n] == s_arg[n]) ++n;
         n_acc[row] = n;
@@ -157,36 +188,39 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     const uint32_t k0 = (uint32_t)seed, k1 = (uint32_t)(seed >> 32);
     const uint32_t c2 = (uint32_t)step, c3 = (uint32_t)(step >> 32);
     const double T = (double)temperature;
-    int n = k;
-    for (int i = 0; i < k; ++i) {
+    // ---- the accept tests of all positions at once (thread i: position i)
+    for (int i = threadIdx.x; i < k; i += blockDim.x) {
         int x = tok[i];
-        Philox4 r = philox4x32_10((uint32_t)i, (uint32_t)row, c2, c3, k0, k1);
+        const Philox4 r = philox4x32_10((uint32_t)i, (uint32_t)row, c2, c3, k0, k1);
         const bool point = dl == nullptr || (onehot && onehot[(long long)row * k + i] != 0);
         bool accept = false;
         if (x < 0 || x >= V) {
             set_status(status, CSD_ERR_BAD_TOKEN);
             x = 0;
         } else {
-            double u = word_uniform(r.w[0]);
-            double px = exp(((double)tl[((long long)row * (k + 1) + i) * V + x] - (double)s_mx[i]) / T) / (double)s_z[i];
+            const double u = word_uniform(r.w[0]);
+            const double px = exp(((double)tl[((long long)row * (k + 1) + i) * V + x] - (double)s_mx[i]) / T) / (double)s_z[i];
             double qx = 1.0;
             if (!point)
                 qx = exp(((double)dl[((long long)row * k + i) * V + x] - (double)s_mx[k + 1 + i]) / T) /
                      (double)s_z[k + 1 + i];
             accept = u * qx < (double)lenience * px;
         }
-        if (!accept) {
-            n = i;
-            ri.mode = point ? MODE_RESID_POINT : MODE_RESID_LOGITS;
-            ri.x = x;
-            ri.max_t = (double)s_mx[i];
-            ri.max_q = point ? 0.0 : (double)s_mx[k + 1 + i];
-            ri.u2 = word_uniform(r.w[1]);
-            break;
-        }
+        s_acc[i] = accept ? 1 : 0; s_x[i] = x; s_point[i] = point ? 1 : 0; s_u2[i] = word_uniform(r.w[1]);
     }
-    if (n == k) {
-        Philox4 r = philox4x32_10((uint32_t)k, (uint32_t)row, c2, c3, k0, k1);
+    __syncthreads();
+    if (threadIdx.x != 0) return;
+    int n = 0;
+    while (n < k && s_acc[n]) ++n;
+    if (n < k) {
+        const bool point = s_point[n] != 0;
+        ri.mode = point ? MODE_RESID_POINT : MODE_RESID_LOGITS;
+        ri.x = s_x[n];
+        ri.max_t = (double)s_mx[n];
+        ri.max_q = point ? 0.0 : (double)s_mx[k + 1 + n];
+        ri.u2 = s_u2[n];
+    } else {
+        const Philox4 r = philox4x32_10((uint32_t)k, (uint32_t)row, c2, c3, k0, k1);
         ri.mode = MODE_TARGET_ONLY;
         ri.max_t = (double)s_mx[k];
         ri.u2 = word_uniform(r.w[1]);
@@ -197,10 +231,10 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
 }
 
 // ---------------------------------------------------------------------------------------------
-// resample passes (fp64).  grid = (rows, chunks)
+// resample passes (fp64).  grid = (rows, chunks).  Every sum has one fixed order: lanes by
+// xor-shuffle, warps in index order, chunks in index order.
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ double block_sum_ordered(double v, double* s_warp) {
-    // fixed reduction tree: lanes by xor-shuffle, then warps in index order
     v = warp_sum(v);
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     __syncthreads();
@@ -211,6 +245,44 @@ __device__ __forceinline__ double block_sum_ordered(double v, double* s_warp) {
     return tot;
 }
 
+// exp(x) for x <= 0 in fp64: x = n ln2 + r with |r| <= ln2 / 2, e^r by its Taylor series to r^11
+// (remainder below 2.3e-13 relative), times 2^n through the exponent field.  Below -708 the
+// result is 0 (the true value is under the smallest normal number).
+__device__ __forceinline__ double exp_neg(double x) {
+    if (!(x > -708.0)) return 0.0;
+    const double n = rint(x * 1.4426950408889634);
+    double r = fma(-n, 6.93147180369123816490e-01, x);        // ln 2, high part (low bits clear)
+    r = fma(-n, 1.90821492927058770002e-10, r);               // ln 2, low part
+    double p = 1.0 / 39916800.0;
+    p = fma(p, r, 1.0 / 3628800.0);
+    p = fma(p, r, 1.0 / 362880.0);
+    p = fma(p, r, 1.0 / 40320.0);
+    p = fma(p, r, 1.0 / 5040.0);
+    p = fma(p, r, 1.0 / 720.0);
+    p = fma(p, r, 1.0 / 120.0);
+    p = fma(p, r, 1.0 / 24.0);
+    p = fma(p, r, 1.0 / 6.0);
+    p = fma(p, r, 0.5);
+    p = fma(p, r, 1.0);
+    p = fma(p, r, 1.0);
+    const long long bits = __double_as_longlong(p) + ((long long)n << 52);   // n >= -1022: stays a normal number
+    return __longlong_as_double(bits);
+}
+
+struct ResidualCtx {
+    const float* t; const float* d;
+    double max_t, max_q, invT, inv_zt, inv_zq;
+    int mode, x;
+};
+__device__ __forceinline__ double residual_at(const ResidualCtx& c, int e) {
+    const double p = exp_neg(((double)c.t[e] - c.max_t) * c.invT) * c.inv_zt;
+    if (c.mode == MODE_TARGET_ONLY) return p;
+    const double q = c.mode == MODE_RESID_POINT ? (e == c.x ? 1.0 : 0.0)
+                                                : exp_neg(((double)c.d[e] - c.max_q) * c.invT) * c.inv_zq;
+    const double r = p - q;
+    return r > 0.0 ? r : 0.0;
+}
+
 // pass 1: per-chunk sums of exp((t - max_t)/T) and exp((d - max_q)/T)
 __global__ void __launch_bounds__(RS_THREADS)
 resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
@@ -219,17 +291,17 @@ resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, in
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
-    const double T = (double)temperature;
+    const double invT = 1.0 / (double)temperature;
     const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
     const float* d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
     const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
     double sp = 0.0, sq = 0.0;
 #pragma unroll
     for (int j = 0; j < RS_PER_THREAD; ++j) {
-        int e = e0 + j;
+        const int e = e0 + j;
         if (e < V) {
-            sp += exp(((double)t[e] - ri.max_t) / T);
-            if (d) sq += exp(((double)d[e] - ri.max_q) / T);
+            sp += exp_neg(((double)t[e] - ri.max_t) * invT);
+            if (d) sq += exp_neg(((double)d[e] - ri.max_q) * invT);
         }
     }
     sp = block_sum_ordered(sp, s_warp);
@@ -237,109 +309,93 @@ resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, in
     if (threadIdx.x == 0) zpart[(long long)row * nchunk + chunk] = make_double2(sp, sq);
 }
 
-__device__ __forceinline__ double residual_value(double ep, double eq, double Zp, double Zq, int mode, int e, int x) {
-    double p = ep / Zp;
-    if (mode == MODE_TARGET_ONLY) return p;
-    double q = mode == MODE_RESID_POINT ? (e == x ? 1.0 : 0.0) : eq / Zq;
-    double r = p - q;
-    return r > 0.0 ? r : 0.0;
-}
-
-// pass 2: per-chunk mass of the residual
+// pass 2: per-chunk mass of the residual; the CTA that arrives last at the row's ticket picks the token
 __global__ void __launch_bounds__(RS_THREADS)
-resample_mass_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
-                     const RowInfo* __restrict__ info, const double2* __restrict__ zpart,
-                     double* __restrict__ rpart, int nchunk) {
+resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
+                     const RowInfo* __restrict__ info, const double2* __restrict__ zpart, double* __restrict__ rpart,
+                     unsigned* __restrict__ tickets, int nchunk, int* __restrict__ out_tok) {
     const int row = blockIdx.x, chunk = blockIdx.y;
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
-    __shared__ double s_Z[2];
+    __shared__ double s_scan[RS_THREADS / 32];
+    __shared__ double s_d[4];    // Zp, Zq, target, base
+    __shared__ int s_i[3];       // chunk, mode, forced-last flag
+    __shared__ int s_pick, s_last, s_is_last;
+    const double2* zrow = zpart + (long long)row * nchunk;
+    double* rrow = rpart + (long long)row * nchunk;
     if (threadIdx.x == 0) {
         double Zp = 0.0, Zq = 0.0;
         for (int c = 0; c < nchunk; ++c) {
-            double2 z = zpart[(long long)row * nchunk + c];
+            const double2 z = zrow[c];
             Zp += z.x; Zq += z.y;
         }
-        s_Z[0] = Zp; s_Z[1] = Zq;
+        s_d[0] = Zp; s_d[1] = Zq;
     }
     __syncthreads();
-    const double Zp = s_Z[0], Zq = s_Z[1], T = (double)temperature;
-    const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
-    const float* d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
-    const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
-    double s = 0.0;
+    const double Zp = s_d[0], Zq = s_d[1];
+    ResidualCtx c;
+    c.t = tl + ((long long)row * (k + 1) + ri.n) * V;
+    c.d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
+    c.max_t = ri.max_t; c.max_q = ri.max_q; c.invT = 1.0 / (double)temperature;
+    c.inv_zt = 1.0 / Zp; c.inv_zq = Zq > 0.0 ? 1.0 / Zq : 0.0;
+    c.mode = ri.mode; c.x = ri.x;
+    {
+        const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
+        double sr = 0.0;
 #pragma unroll
-    for (int j = 0; j < RS_PER_THREAD; ++j) {
-        int e = e0 + j;
-        if (e < V) {
-            double ep = exp(((double)t[e] - ri.max_t) / T);
-            double eq = d ? exp(((double)d[e] - ri.max_q) / T) : 0.0;
-            s += residual_value(ep, eq, Zp, Zq, ri.mode, e, ri.x);
+        for (int j = 0; j < RS_PER_THREAD; ++j)
+            if (e0 + j < V) sr += residual_at(c, e0 + j);
+        sr = block_sum_ordered(sr, s_warp);
+        if (threadIdx.x == 0) {
+            rrow[chunk] = sr;
+            __threadfence();
+            s_is_last = atomicAdd(&tickets[row], 1u) == (unsigned)nchunk - 1u;
         }
+        __syncthreads();
+        if (!s_is_last) return;
+        __threadfence();
     }
-    s = block_sum_ordered(s, s_warp);
-    if (threadIdx.x == 0) rpart[(long long)row * nchunk + chunk] = s;
-}
-
-// pass 3: one CTA per row picks the token
-__global__ void __launch_bounds__(RS_THREADS)
-resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
-                     const RowInfo* __restrict__ info, const double2* __restrict__ zpart,
-                     const double* __restrict__ rpart, int nchunk, int* __restrict__ out_tok) {
-    const int row = blockIdx.x;
-    const RowInfo ri = info[row];
-    if (ri.mode == MODE_DONE) return;
-    __shared__ double s_d[4];   // Zp, Zq, target, base
-    __shared__ int s_i[3];      // chunk, mode, forced-last flag
-    __shared__ double s_scan[RS_THREADS / 32];
-    __shared__ int s_pick, s_last;
+    // ---- last CTA of the row: which chunk holds u2 * S, then the entry inside it
     if (threadIdx.x == 0) {
-        double Zp = 0.0, Zq = 0.0, S = 0.0;
-        for (int c = 0; c < nchunk; ++c) {
-            double2 z = zpart[(long long)row * nchunk + c];
-            Zp += z.x; Zq += z.y;
-            S += rpart[(long long)row * nchunk + c];
-        }
+        double S = 0.0;
+        for (int ch = 0; ch < nchunk; ++ch) S += __ldcg(rrow + ch);
         int mode = ri.mode;
         const bool empty = !(S > 0.0) || !isfinite(S);
         if (empty) {   // empty residual: fall back to the target law itself
             mode = MODE_TARGET_ONLY;
             S = 0.0;
-            for (int c = 0; c < nchunk; ++c) S += zpart[(long long)row * nchunk + c].x / Zp;
+            for (int ch = 0; ch < nchunk; ++ch) S += zrow[ch].x * c.inv_zt;
         }
         const double target = ri.u2 * S;
         double cum = 0.0, base = 0.0;
-        int chunk = -1, last_pos = 0;
-        for (int c = 0; c < nchunk; ++c) {
-            double mass = empty ? zpart[(long long)row * nchunk + c].x / Zp : rpart[(long long)row * nchunk + c];
-            if (mass > 0.0) last_pos = c;
-            if (cum + mass > target) { chunk = c; base = cum; break; }
+        int pick_chunk = -1, last_pos = 0;
+        for (int ch = 0; ch < nchunk; ++ch) {
+            const double mass = empty ? zrow[ch].x * c.inv_zt : __ldcg(rrow + ch);
+            if (mass > 0.0) last_pos = ch;
+            if (cum + mass > target) { pick_chunk = ch; base = cum; break; }
             cum += mass;
         }
         int forced = 0;
-        if (chunk < 0) { chunk = last_pos; forced = 1; }
-        s_d[0] = Zp; s_d[1] = Zq; s_d[2] = target; s_d[3] = base;
-        s_i[0] = chunk; s_i[1] = mode; s_i[2] = forced;
+        if (pick_chunk < 0) { pick_chunk = last_pos; forced = 1; }
+        s_d[2] = target; s_d[3] = base;
+        s_i[0] = pick_chunk; s_i[1] = mode; s_i[2] = forced;
         s_pick = 0x7fffffff; s_last = -1;
     }
     __syncthreads();
-    const double Zp = s_d[0], Zq = s_d[1], target = s_d[2], base = s_d[3], T = (double)temperature;
-    const int chunk = s_i[0], mode = s_i[1], forced = s_i[2];
-    const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
-    const float* d = mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
-    const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
+    const double target = s_d[2], base = s_d[3];
+    const int pick_chunk = s_i[0], forced = s_i[2];
+    c.mode = s_i[1];
+    const int e0 = pick_chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
     double r[RS_PER_THREAD];
     double local = 0.0;
     int my_last = -1;
 #pragma unroll
     for (int j = 0; j < RS_PER_THREAD; ++j) {
-        int e = e0 + j;
+        const int e = e0 + j;
         r[j] = 0.0;
         if (e < V) {
-            double ep = exp(((double)t[e] - ri.max_t) / T);
-            double eq = d ? exp(((double)d[e] - ri.max_q) / T) : 0.0;
-            r[j] = residual_value(ep, eq, Zp, Zq, mode, e, ri.x);
+            r[j] = residual_at(c, e);
             if (r[j] > 0.0) my_last = e;
         }
         local += r[j];
@@ -349,7 +405,7 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     double incl = local;
 #pragma unroll
     for (int o = 1; o < 32; o <<= 1) {
-        double up = __shfl_up_sync(0xffffffffu, incl, o);
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
         if (lane >= o) incl += up;
     }
     if (lane == 31) s_scan[warp] = incl;
@@ -368,14 +424,11 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     if (found != 0x7fffffff) atomicMin(&s_pick, found);
     if (my_last >= 0) atomicMax(&s_last, my_last);
     __syncthreads();
-    if (threadIdx.x == 0) {
-        int pick = s_pick != 0x7fffffff ? s_pick : (s_last >= 0 ? s_last : 0);
-        out_tok[row] = pick;
-    }
+    if (threadIdx.x == 0) out_tok[row] = s_pick != 0x7fffffff ? s_pick : (s_last >= 0 ? s_last : 0);
 }
 
 struct AcceptLayout {
-    size_t part_off, info_off, z_off, r_off, total;
+    size_t part_off, info_off, z_off, r_off, ticket_off, total;
     int nchunk_a, nchunk_r;
 };
 
@@ -385,12 +438,65 @@ static AcceptLayout accept_layout(int rows, int k, int V) {
     L.nchunk_r = (V + RS_CHUNK - 1) / RS_CHUNK;
     size_t nvec = (size_t)rows * (2 * (size_t)k + 1);
     size_t off = 0;
-    L.part_off = off; off = align_up(off + nvec * L.nchunk_a * sizeof(StatPartial), 256);
-    L.info_off = off; off = align_up(off + (size_t)rows * sizeof(RowInfo), 256);
-    L.z_off = off;    off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double2), 256);
-    L.r_off = off;    off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double), 256);
+    L.part_off = off;   off = align_up(off + nvec * L.nchunk_a * sizeof(StatPartial), 256);
+    L.info_off = off;   off = align_up(off + (size_t)rows * sizeof(RowInfo), 256);
+    L.z_off = off;      off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double2), 256);
+    L.r_off = off;      off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double), 256);
+    L.ticket_off = off; off = align_up(off + (size_t)rows * sizeof(unsigned), 256);
     L.total = off;
     return L;
+}
+
+static int accept_sm_count() {
+    static int n = 0;
+    if (n == 0) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess ||
+            cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess || n <= 0)
+            n = 148;
+    }
+    return n;
+}
+
+// The three passes on scratch `ws` (accept_layout bytes).  Every word a pass reads is written by an
+// earlier pass of the same call (the decide pass clears the resample tickets), so the scratch
+// needs no initialisation.
+static csd_status run_accept(const float* tl, const float* dl_in, const int32_t* onehot, const int32_t* tokens, int rows,
+                             int k, int V, float temperature, float lenience, uint64_t seed, uint64_t step,
+                             int32_t* n_acc, int32_t* out_tok, char* ws, const AcceptLayout& L, int* status,
+                             cudaStream_t st) {
+    StatPartial* part = (StatPartial*)(ws + L.part_off);
+    RowInfo* info = (RowInfo*)(ws + L.info_off);
+    double2* zpart = (double2*)(ws + L.z_off);
+    double* rpart = (double*)(ws + L.r_off);
+    unsigned* tickets = (unsigned*)(ws + L.ticket_off);
+    const bool greedy = temperature == 0.f;
+    const float invT = greedy ? 1.f : 1.f / temperature;
+    const bool use_d = dl_in != nullptr && k > 0 && !greedy;
+    const float* dl = use_d ? dl_in : nullptr;
+    const long long n_tvec = (long long)rows * (k + 1);
+    const long long nvec = n_tvec + (use_d ? (long long)rows * k : 0);
+    if (nvec > 0x7fffffffLL) return CSD_ERR_UNSUPPORTED;
+    const bool vec_ok = (V % 4 == 0) && (((uintptr_t)tl & 15) == 0) && (!use_d || ((uintptr_t)dl & 15) == 0);
+    const long long items = nvec * L.nchunk_a;
+    long long ctas = (items + ST_THREADS / 32 - 1) / (ST_THREADS / 32);
+    const long long cap = (long long)accept_sm_count() * 2;       // two resident CTAs per SM, grid-stride beyond
+    if (ctas > cap) ctas = cap;
+    if (vec_ok)
+        accept_stats_kernel<true><<<(unsigned)ctas, ST_THREADS, 0, st>>>(tl, dl, n_tvec, V, invT, greedy, part, L.nchunk_a, items);
+    else
+        accept_stats_kernel<false><<<(unsigned)ctas, ST_THREADS, 0, st>>>(tl, dl, n_tvec, V, invT, greedy, part, L.nchunk_a, items);
+    accept_decide_kernel<<<rows, 128, 0, st>>>(tl, dl, onehot, tokens, rows, k, V, temperature, lenience, seed, step, part,
+                                               L.nchunk_a, n_acc, out_tok, info, tickets, status);
+    count_launch(2);
+    if (!greedy) {
+        dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
+        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, L.nchunk_r);
+        resample_pick_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, rpart, tickets, L.nchunk_r, out_tok);
+        count_launch(2);
+    }
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
 }
 
 }  // namespace csd
@@ -415,43 +521,11 @@ extern "C" csd_status csd_spec_accept(const float* target_logits_dev, const floa
     if (((uintptr_t)workspace_dev & 255) != 0) return CSD_ERR_INVALID_ARG;
     const AcceptLayout L = accept_layout(rows, k, V);
     if (workspace_bytes < L.total) return CSD_ERR_CAPACITY;
-    if (L.nchunk_a > 65535 || L.nchunk_r > 65535) return CSD_ERR_UNSUPPORTED;
-    cudaStream_t st = (cudaStream_t)stream;
+    if (L.nchunk_r > 65535) return CSD_ERR_UNSUPPORTED;
     int* status = status_word_device();
     if (!status) return CSD_ERR_CUDA;
-    char* ws = (char*)workspace_dev;
-    StatPartial* part = (StatPartial*)(ws + L.part_off);
-    RowInfo* info = (RowInfo*)(ws + L.info_off);
-    double2* zpart = (double2*)(ws + L.z_off);
-    double* rpart = (double*)(ws + L.r_off);
-    const bool greedy = temperature == 0.f;
-    const float invT = greedy ? 1.f : 1.f / temperature;
-    const bool use_d = draft_logits_dev != nullptr && k > 0 && !greedy;
-    const float* dl = use_d ? draft_logits_dev : nullptr;
-    const long long n_tvec = (long long)rows * (k + 1);
-    const long long nvec = n_tvec + (use_d ? (long long)rows * k : 0);
-    if (nvec > 0x7fffffffLL) return CSD_ERR_UNSUPPORTED;
-    const bool vec_ok = (V % 4 == 0) && (((uintptr_t)target_logits_dev & 15) == 0) &&
-                        (!use_d || ((uintptr_t)draft_logits_dev & 15) == 0);
-    dim3 grid((unsigned)nvec, (unsigned)L.nchunk_a);
-    if (vec_ok)
-        accept_stats_kernel<true><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
-    else
-        accept_stats_kernel<false><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
-    accept_decide_kernel<<<rows, 128, 0, st>>>(target_logits_dev, dl, onehot_dev, draft_tokens_dev, rows, k, V,
-                                               temperature, lenience, seed, step, part, L.nchunk_a,
-                                               n_accepted_dev, out_token_dev, info, status);
-    count_launch(2);
-    if (!greedy) {
-        dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
-        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, L.nchunk_r);
-        resample_mass_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart, L.nchunk_r);
-        resample_pick_kernel<<<rows, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart,
-                                                          L.nchunk_r, out_token_dev);
-        count_launch(3);
-    }
-    CSD_CUDA(cudaGetLastError());
-    return CSD_OK;
+    return run_accept(target_logits_dev, draft_logits_dev, onehot_dev, draft_tokens_dev, rows, k, V, temperature, lenience,
+                      seed, step, n_accepted_dev, out_token_dev, (char*)workspace_dev, L, status, (cudaStream_t)stream);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -479,7 +553,7 @@ extern "C" csd_status csd_spec_accept_static(const float* target_logits_dev, con
     if (k > 0 && !draft_tokens_dev) return CSD_ERR_INVALID_ARG;
     const AcceptLayout L = accept_layout(rows, k, V);
     if (L.total > STATIC_SCRATCH_BYTES) return CSD_ERR_CAPACITY;   // the problem does not fit the fixed scratch
-    if (L.nchunk_a > 65535 || L.nchunk_r > 65535) return CSD_ERR_UNSUPPORTED;
+    if (L.nchunk_r > 65535) return CSD_ERR_UNSUPPORTED;
     // Set-up, once per device: in host code the array's name is only a handle, so ask the runtime
     // for the address the kernels can use.  Nothing is allocated here.
     int dev = 0;
@@ -495,39 +569,7 @@ extern "C" csd_status csd_spec_accept_static(const float* target_logits_dev, con
         }
         ws = (char*)g_accept_scratch_ptr[dev];
     }
-    cudaStream_t st = (cudaStream_t)stream;
-    StatPartial* part = (StatPartial*)(ws + L.part_off);
-    RowInfo* info = (RowInfo*)(ws + L.info_off);
-    double2* zpart = (double2*)(ws + L.z_off);
-    double* rpart = (double*)(ws + L.r_off);
-    const bool greedy = temperature == 0.f;
-    const float invT = greedy ? 1.f : 1.f / temperature;
-    const bool use_d = draft_logits_dev != nullptr && k > 0 && !greedy;
-    const float* dl = use_d ? draft_logits_dev : nullptr;
-    const long long n_tvec = (long long)rows * (k + 1);
-    const long long nvec = n_tvec + (use_d ? (long long)rows * k : 0);
-    if (nvec > 0x7fffffffLL) return CSD_ERR_UNSUPPORTED;
-    const bool vec_ok = (V % 4 == 0) && (((uintptr_t)target_logits_dev & 15) == 0) &&
-                        (!use_d || ((uintptr_t)draft_logits_dev & 15) == 0);
-    // Every word of the scratch that a pass reads is written by an earlier pass of the same call,
-    // so nothing has to be cleared even though the array still holds the previous call's data.
-    dim3 grid((unsigned)nvec, (unsigned)L.nchunk_a);
-    if (vec_ok)
-        accept_stats_kernel<true><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
-    else
-        accept_stats_kernel<false><<<grid, ST_THREADS, 0, st>>>(target_logits_dev, dl, n_tvec, V, invT, greedy, part, L.nchunk_a);
-    accept_decide_kernel<<<rows, 128, 0, st>>>(target_logits_dev, dl, onehot_dev, draft_tokens_dev, rows, k, V,
-                                               temperature, lenience, seed, step, part, L.nchunk_a,
-                                               n_accepted_dev, out_token_dev, info, nullptr);
-    count_launch(2);
-    if (!greedy) {
-        dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
-        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, L.nchunk_r);
-        resample_mass_kernel<<<g2, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart, L.nchunk_r);
-        resample_pick_kernel<<<rows, RS_THREADS, 0, st>>>(target_logits_dev, dl, k, V, temperature, info, zpart, rpart,
-                                                          L.nchunk_r, out_token_dev);
-        count_launch(3);
-    }
-    CSD_CUDA(cudaGetLastError());
-    return CSD_OK;
+    // (bad token ids are not recorded in the status word here: looking that word up may allocate)
+    return run_accept(target_logits_dev, draft_logits_dev, onehot_dev, draft_tokens_dev, rows, k, V, temperature, lenience,
+                      seed, step, n_accepted_dev, out_token_dev, ws, L, nullptr, (cudaStream_t)stream);
 }
