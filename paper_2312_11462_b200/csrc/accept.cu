@@ -170,7 +170,7 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
         }
         s_mx[i] = mx; s_z[i] = greedy ? 0.f : z; s_arg[i] = arg;
     }
-    if (threadIdx.x == 0 && tickets) tickets[row] = 0u;     // for the resample pass that follows
+    if (threadIdx.x == 0 && tickets) { tickets[row] = 0u; tickets[rows + row] = 0u; }   // for the two resample passes
     __syncthreads();
     const int* tok = tokens + (long long)row * k;
     RowInfo ri;
@@ -286,7 +286,8 @@ __device__ __forceinline__ double residual_at(const ResidualCtx& c, int e) {
 // pass 1: per-chunk sums of exp((t - max_t)/T) and exp((d - max_q)/T)
 __global__ void __launch_bounds__(RS_THREADS)
 resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
-                  const RowInfo* __restrict__ info, double2* __restrict__ zpart, int nchunk) {
+                  const RowInfo* __restrict__ info, double2* __restrict__ zpart, double2* __restrict__ zsum,
+                  unsigned* __restrict__ tickets, int nchunk) {
     const int row = blockIdx.x, chunk = blockIdx.y;
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
@@ -306,34 +307,47 @@ resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, in
     }
     sp = block_sum_ordered(sp, s_warp);
     sq = block_sum_ordered(sq, s_warp);
-    if (threadIdx.x == 0) zpart[(long long)row * nchunk + chunk] = make_double2(sp, sq);
+    __shared__ int s_is_last;
+    __shared__ double2 s_z[RS_THREADS];
+    double2* zrow = zpart + (long long)row * nchunk;
+    if (threadIdx.x == 0) {
+        zrow[chunk] = make_double2(sp, sq);
+        __threadfence();
+        s_is_last = atomicAdd(&tickets[row], 1u) == (unsigned)nchunk - 1u;
+    }
+    __syncthreads();
+    if (!s_is_last) return;
+    // last chunk of the row: the totals, summed in chunk order (loads in parallel, adds by one thread)
+    __threadfence();
+    double Zp = 0.0, Zq = 0.0;
+    for (int c0 = 0; c0 < nchunk; c0 += RS_THREADS) {
+        const int c = c0 + threadIdx.x;
+        s_z[threadIdx.x] = c < nchunk ? make_double2(__ldcg(&zrow[c].x), __ldcg(&zrow[c].y)) : make_double2(0.0, 0.0);
+        __syncthreads();
+        if (threadIdx.x == 0)
+            for (int i = 0; i < RS_THREADS && c0 + i < nchunk; ++i) { Zp += s_z[i].x; Zq += s_z[i].y; }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) zsum[row] = make_double2(Zp, Zq);
 }
 
 // pass 2: per-chunk mass of the residual; the CTA that arrives last at the row's ticket picks the token
 __global__ void __launch_bounds__(RS_THREADS)
 resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
-                     const RowInfo* __restrict__ info, const double2* __restrict__ zpart, double* __restrict__ rpart,
-                     unsigned* __restrict__ tickets, int nchunk, int* __restrict__ out_tok) {
+                     const RowInfo* __restrict__ info, const double2* __restrict__ zpart,
+                     const double2* __restrict__ zsum, double* __restrict__ rpart, unsigned* __restrict__ tickets,
+                     int nchunk, int* __restrict__ out_tok) {
     const int row = blockIdx.x, chunk = blockIdx.y;
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
     __shared__ double s_scan[RS_THREADS / 32];
-    __shared__ double s_d[4];    // Zp, Zq, target, base
+    __shared__ double s_d[2];    // target, base
     __shared__ int s_i[3];       // chunk, mode, forced-last flag
     __shared__ int s_pick, s_last, s_is_last;
     const double2* zrow = zpart + (long long)row * nchunk;
     double* rrow = rpart + (long long)row * nchunk;
-    if (threadIdx.x == 0) {
-        double Zp = 0.0, Zq = 0.0;
-        for (int c = 0; c < nchunk; ++c) {
-            const double2 z = zrow[c];
-            Zp += z.x; Zq += z.y;
-        }
-        s_d[0] = Zp; s_d[1] = Zq;
-    }
-    __syncthreads();
-    const double Zp = s_d[0], Zq = s_d[1];
+    const double Zp = zsum[row].x, Zq = zsum[row].y;
     ResidualCtx c;
     c.t = tl + ((long long)row * (k + 1) + ri.n) * V;
     c.d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
@@ -356,34 +370,56 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
         if (!s_is_last) return;
         __threadfence();
     }
-    // ---- last CTA of the row: which chunk holds u2 * S, then the entry inside it
-    if (threadIdx.x == 0) {
-        double S = 0.0;
-        for (int ch = 0; ch < nchunk; ++ch) S += __ldcg(rrow + ch);
-        int mode = ri.mode;
-        const bool empty = !(S > 0.0) || !isfinite(S);
-        if (empty) {   // empty residual: fall back to the target law itself
-            mode = MODE_TARGET_ONLY;
-            S = 0.0;
-            for (int ch = 0; ch < nchunk; ++ch) S += zrow[ch].x * c.inv_zt;
-        }
-        const double target = ri.u2 * S;
-        double cum = 0.0, base = 0.0;
+    // ---- last CTA of the row: which chunk holds u2 * S, then the entry inside it.  Chunk masses are
+    //      fetched by all threads into shared memory; one thread adds them in chunk order.
+    __shared__ double s_mass[RS_THREADS];
+    __shared__ double s_S;
+    __shared__ int s_empty;
+    for (int pass = 0; pass < 2; ++pass) {
+        // pass 0: total mass S (and whether the residual is empty); pass 1: the chunk that holds u2 * S
+        const bool empty = pass == 1 && s_empty;
+        double acc = 0.0, target = 0.0;
         int pick_chunk = -1, last_pos = 0;
-        for (int ch = 0; ch < nchunk; ++ch) {
-            const double mass = empty ? zrow[ch].x * c.inv_zt : __ldcg(rrow + ch);
-            if (mass > 0.0) last_pos = ch;
-            if (cum + mass > target) { pick_chunk = ch; base = cum; break; }
-            cum += mass;
+        double base = 0.0;
+        if (pass == 1) target = ri.u2 * s_S;
+        for (int c0 = 0; c0 < nchunk; c0 += RS_THREADS) {
+            const int ch = c0 + threadIdx.x;
+            double mval = 0.0;
+            if (ch < nchunk) mval = empty ? zrow[ch].x * c.inv_zt : __ldcg(rrow + ch);
+            s_mass[threadIdx.x] = mval;
+            __syncthreads();
+            if (threadIdx.x == 0) {
+                for (int i = 0; i < RS_THREADS && c0 + i < nchunk; ++i) {
+                    const double mass = s_mass[i];
+                    if (pass == 0) { acc += mass; continue; }
+                    if (pick_chunk >= 0) break;
+                    if (mass > 0.0) last_pos = c0 + i;
+                    if (acc + mass > target) { pick_chunk = c0 + i; base = acc; break; }
+                    acc += mass;
+                }
+            }
+            __syncthreads();
         }
-        int forced = 0;
-        if (pick_chunk < 0) { pick_chunk = last_pos; forced = 1; }
-        s_d[2] = target; s_d[3] = base;
-        s_i[0] = pick_chunk; s_i[1] = mode; s_i[2] = forced;
-        s_pick = 0x7fffffff; s_last = -1;
+        if (threadIdx.x == 0) {
+            if (pass == 0) {
+                const bool is_empty = !(acc > 0.0) || !isfinite(acc);
+                s_empty = is_empty ? 1 : 0;
+                if (is_empty) {   // empty residual: fall back to the target law itself
+                    acc = 0.0;
+                    for (int ch = 0; ch < nchunk; ++ch) acc += zrow[ch].x * c.inv_zt;
+                }
+                s_S = acc;
+            } else {
+                int forced = 0;
+                if (pick_chunk < 0) { pick_chunk = last_pos; forced = 1; }
+                s_d[0] = target; s_d[1] = base;
+                s_i[0] = pick_chunk; s_i[1] = s_empty ? (int)MODE_TARGET_ONLY : ri.mode; s_i[2] = forced;
+                s_pick = 0x7fffffff; s_last = -1;
+            }
+        }
+        __syncthreads();
     }
-    __syncthreads();
-    const double target = s_d[2], base = s_d[3];
+    const double target = s_d[0], base = s_d[1];
     const int pick_chunk = s_i[0], forced = s_i[2];
     c.mode = s_i[1];
     const int e0 = pick_chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
@@ -428,7 +464,7 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
 }
 
 struct AcceptLayout {
-    size_t part_off, info_off, z_off, r_off, ticket_off, total;
+    size_t part_off, info_off, z_off, zsum_off, r_off, ticket_off, total;
     int nchunk_a, nchunk_r;
 };
 
@@ -442,7 +478,8 @@ static AcceptLayout accept_layout(int rows, int k, int V) {
     L.info_off = off;   off = align_up(off + (size_t)rows * sizeof(RowInfo), 256);
     L.z_off = off;      off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double2), 256);
     L.r_off = off;      off = align_up(off + (size_t)rows * L.nchunk_r * sizeof(double), 256);
-    L.ticket_off = off; off = align_up(off + (size_t)rows * sizeof(unsigned), 256);
+    L.zsum_off = off;   off = align_up(off + (size_t)rows * sizeof(double2), 256);
+    L.ticket_off = off; off = align_up(off + 2 * (size_t)rows * sizeof(unsigned), 256);   // normaliser pass, mass pass
     L.total = off;
     return L;
 }
@@ -469,6 +506,7 @@ static csd_status run_accept(const float* tl, const float* dl_in, const int32_t*
     RowInfo* info = (RowInfo*)(ws + L.info_off);
     double2* zpart = (double2*)(ws + L.z_off);
     double* rpart = (double*)(ws + L.r_off);
+    double2* zsum = (double2*)(ws + L.zsum_off);
     unsigned* tickets = (unsigned*)(ws + L.ticket_off);
     const bool greedy = temperature == 0.f;
     const float invT = greedy ? 1.f : 1.f / temperature;
@@ -491,8 +529,8 @@ static csd_status run_accept(const float* tl, const float* dl_in, const int32_t*
     count_launch(2);
     if (!greedy) {
         dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
-        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, L.nchunk_r);
-        resample_pick_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, rpart, tickets, L.nchunk_r, out_tok);
+        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, tickets, L.nchunk_r);
+        resample_pick_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, rpart, tickets + rows, L.nchunk_r, out_tok);
         count_launch(2);
     }
     CSD_CUDA(cudaGetLastError());
