@@ -313,6 +313,19 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
             __syncwarp();
             if (lane == 0) mbar_arrive(&ctl->acc_empty[b]);
             const int col = q * 32 + lane, n = tile * TILE_N + col;
+            // what the finishing step needs besides the sums is requested now, so that it travels while
+            // the partial sums are parked and the ticket is taken (only the finisher uses it)
+            float yold[M];
+            float out_g = 1.f;
+#pragma unroll
+            for (int r = 0; r < M; ++r) yold[r] = 0.f;
+            if (n < p.N) {
+                if (p.epilogue == EPI_ADD) {
+#pragma unroll
+                    for (int r = 0; r < M; ++r) yold[r] = __ldcg(p.Y + (size_t)r * p.ldy + n);
+                }
+                if (p.out_xs && p.out_gain) out_g = __bfloat162float(p.out_gain[n]);
+            }
             if (seg_len < p.nkb) {
                 // part of a tile: leave it in this CTA's slot (0 = the CTA's first segment, 1 = a later
                 // one); the CTA that arrives last adds all parts in CTA order and finishes the tile
@@ -338,17 +351,18 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 for (int u = 0; u < NT; ++u)
 #pragma unroll
                     for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
-                // parts in CTA order, a few contributors' loads in flight at a time
-                constexpr int CH = NT * M <= 12 ? 4 : (NT * M <= 24 ? 2 : 1);
+                // parts in CTA order; as many contributors' loads in flight together as about 48 registers
+                // hold (all of them, in one round trip, for a 5-row block)
+                constexpr int NV = NT * M, CH = NV <= 6 ? 8 : (48 / NV < 1 ? 1 : 48 / NV);
                 for (int c = c_lo; c <= c_hi; c += CH) {
-                    float part[CH][NT * M];
+                    float part[CH][NV];
 #pragma unroll
                     for (int h = 0; h < CH; ++h) {
                         const int cc = min(c + h, c_hi);
                         const int slot = (int)(unit_begin(cc, units, ctas) / p.nkb) == tile ? 0 : 1;
                         const float* src = p.partial + ((size_t)cc * 2 + slot) * NT * M * TILE_N + col;
 #pragma unroll
-                        for (int v = 0; v < NT * M; ++v) part[h][v] = __ldcg(src + v * TILE_N);
+                        for (int v = 0; v < NV; ++v) part[h][v] = __ldcg(src + v * TILE_N);
                     }
 #pragma unroll
                     for (int h = 0; h < CH; ++h)
@@ -372,7 +386,7 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 }
                 if (n < p.N) {
                     float* y = p.Y + (size_t)r * p.ldy + n;
-                    if (p.epilogue == EPI_ADD) val += *y;
+                    if (p.epilogue == EPI_ADD) val += yold[r];
                     *y = val;
                 } else {
                     val = 0.f;
@@ -387,11 +401,10 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 }
             }
             if (p.out_xs && n < p.N) {            // the rows as three bf16 terms for the GEMM that reads them next
-                const float g = p.out_gain ? __bfloat162float(p.out_gain[n]) : 1.f;
 #pragma unroll
                 for (int r = 0; r < M; ++r) {
                     uint16_t b1, b2, b3;
-                    split3(outv[r] * g, b1, b2, b3);
+                    split3(outv[r] * out_g, b1, b2, b3);
                     uint16_t* o = reinterpret_cast<uint16_t*>(p.out_xs) + n;
                     o[(size_t)r * p.out_ld] = b1;
                     o[(size_t)(M + r) * p.out_ld] = b2;
