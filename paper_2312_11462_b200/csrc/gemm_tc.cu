@@ -34,7 +34,7 @@ int gemm_path() { return g_path; }
 static int npad_for(int m) { int c = 3 * m; return c <= 16 ? 16 : (c <= 32 ? 32 : (c <= 48 ? 48 : 64)); }
 
 struct TcPlan {
-    int npad, tiles, kblocks, grid, stages;
+    int npad, tiles, kblocks, grid, stages;    // kblocks: stages of work per tile (one or two 64-wide K blocks each)
     size_t smem, scratch_floats;
 };
 
@@ -55,12 +55,13 @@ static TcPlan tc_plan(int m, int N, int K, bool dual) {
     p.npad = npad_for(m);
     p.tiles = (N + TILE_N - 1) / TILE_N;
     p.kblocks = (K + KB - 1) / KB;
+    if (!dual) p.kblocks = (p.kblocks + 1) / 2;             // single-matrix GEMM: a stage holds two K blocks
     const long long units = (long long)p.tiles * p.kblocks;
     long long grid = units / 4;                           // at least four units per CTA
     if (grid < 1) grid = 1;
     if (grid > tc_sm_count()) grid = tc_sm_count();
     p.grid = (int)grid;
-    const size_t stage = (size_t)STAGE_BYTES * (dual ? 2 : 1) + (size_t)p.npad * 128;
+    const size_t stage = (size_t)STAGE_BYTES * 2 + (size_t)p.npad * 128 * (dual ? 1 : 2);
     p.stages = (int)((TC_SMEM_MAX - 1024) / stage);
     if (p.stages > 12) p.stages = 12;
     p.smem = (size_t)p.stages * stage + 1024;
@@ -174,7 +175,9 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     constexpr int ACC_COLS = NPAD * NT;                       // tensor-memory columns per accumulator set
     constexpr int TMEM_COLS = 2 * ACC_COLS <= 32 ? 32 : (2 * ACC_COLS <= 64 ? 64 : (2 * ACC_COLS <= 128 ? 128 : 256));
     constexpr int XBYTES = NPAD * 128;                        // the rows' terms for one K block
-    constexpr int STAGE = STAGE_BYTES * NT + XBYTES;
+    constexpr int KS = DUAL ? 1 : 2;                          // K blocks per stage: every stage carries two weight boxes
+    constexpr int WB = 2 * STAGE_BYTES;                       // weight bytes per stage
+    constexpr int STAGE = WB + KS * XBYTES;
     constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(NPAD >> 3) << 17) |
                                ((uint32_t)(TILE_N >> 4) << 24);   // f32 accumulate, bf16 x bf16, K-major both
 
@@ -220,12 +223,17 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
                 unsigned char* dst = ring + (size_t)i * STAGE;
                 mbar_expect_tx(&ctl->full[i], (uint32_t)STAGE);
-                tma_load_2d(dst, &tmW, &ctl->full[i], kb * KB, tile * TILE_N);
+                tma_load_2d(dst, &tmW, &ctl->full[i], kb * KS * KB, tile * TILE_N);
                 if (DUAL) tma_load_2d(dst + STAGE_BYTES, &tmW2, &ctl->full[i], kb * KB, tile * TILE_N);
+                else tma_load_2d(dst + STAGE_BYTES, &tmW, &ctl->full[i], (kb * KS + 1) * KB, tile * TILE_N);   // past K: zero fill
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
-            for (int i = 0; i < pre; ++i)
-                tma_load_2d(ring + (size_t)i * STAGE + STAGE_BYTES * NT, &tmX, &ctl->full[i], (int)((u0 + i) % p.nkb) * KB, 0);
+            for (int i = 0; i < pre; ++i) {
+                const int kb = (int)((u0 + i) % p.nkb);
+#pragma unroll
+                for (int j = 0; j < KS; ++j)
+                    tma_load_2d(ring + (size_t)i * STAGE + WB + j * XBYTES, &tmX, &ctl->full[i], (kb * KS + j) * KB, 0);
+            }
             for (int i = pre; i < items && !*abort_flag; ++i) {
                 const int s = i % p.stages;
                 if (!mbar_wait(&ctl->empty[s], ((i / p.stages) - 1) & 1)) { *abort_flag = 1; break; }
@@ -233,9 +241,12 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
                 unsigned char* dst = ring + (size_t)s * STAGE;
                 mbar_expect_tx(&ctl->full[s], (uint32_t)STAGE);
-                tma_load_2d(dst, &tmW, &ctl->full[s], kb * KB, tile * TILE_N);
+                tma_load_2d(dst, &tmW, &ctl->full[s], kb * KS * KB, tile * TILE_N);
                 if (DUAL) tma_load_2d(dst + STAGE_BYTES, &tmW2, &ctl->full[s], kb * KB, tile * TILE_N);
-                tma_load_2d(dst + STAGE_BYTES * NT, &tmX, &ctl->full[s], kb * KB, 0);
+                else tma_load_2d(dst + STAGE_BYTES, &tmW, &ctl->full[s], (kb * KS + 1) * KB, tile * TILE_N);
+#pragma unroll
+                for (int j = 0; j < KS; ++j)
+                    tma_load_2d(dst + WB + j * XBYTES, &tmX, &ctl->full[s], (kb * KS + j) * KB, 0);
             }
         }
     } else if (warp == 1) {
@@ -254,13 +265,15 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     if (!mbar_wait(&ctl->full[s], (i / p.stages) & 1)) { *abort_flag = 1; break; }
                     tc_fence_after();
                     const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE);
-                    const uint32_t b_addr = a_addr + STAGE_BYTES * NT;
+                    const uint32_t b_addr = a_addr + WB;
 #pragma unroll
-                    for (int k = 0; k < KB / 16; ++k) {
-                        const uint64_t bd = smem_desc_sw128(b_addr + k * 32);
-                        tc_mma(d0, smem_desc_sw128(a_addr + k * 32), bd, IDESC, (j | k) != 0);
-                        if (DUAL) tc_mma(d0 + NPAD, smem_desc_sw128(a_addr + STAGE_BYTES + k * 32), bd, IDESC, (j | k) != 0);
-                    }
+                    for (int h = 0; h < KS; ++h)
+#pragma unroll
+                        for (int k = 0; k < KB / 16; ++k) {
+                            const uint64_t bd = smem_desc_sw128(b_addr + h * XBYTES + k * 32);
+                            tc_mma(d0, smem_desc_sw128(a_addr + h * STAGE_BYTES + k * 32), bd, IDESC, (j | h | k) != 0);
+                            if (DUAL) tc_mma(d0 + NPAD, smem_desc_sw128(a_addr + STAGE_BYTES + k * 32), bd, IDESC, (j | k) != 0);
+                        }
                     tc_commit(&ctl->empty[s]);          // stage reusable once these MMAs have read it
                 }
                 if (*abort_flag) break;
