@@ -235,7 +235,7 @@ csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32
  * cascade, the recursion into level c+1 the vertical cascade.  A review takes at most max_block
  * drafted tokens (surplus drafts are dropped, which keeps the output law).  Lenience applies
  * when a draft reviews, never when the target does.  Each level forwards every token it has not
- * cached yet, in chunks of at most max_block+1 rows (this also serves as prompt prefill).
+ * cached yet, in chunks of at most the model's max_rows rows (this also serves as prompt prefill).
  * Decoder-only models: haystack = prompt, init_seq = prompt.  Encoder-decoder: haystack =
  * encoder input (the encoders are run here), init_seq = decoder start token(s).
  * Host in, host out; the call returns after the stream has finished.

@@ -22,7 +22,7 @@ static CascadeWs cascade_layout(int V, int max_block, int cap, int L, int max_or
     w.seq = put(((size_t)cap + 64) * 4);
     w.hay = put((size_t)(L > 0 ? L : 1) * 4);
     w.mag = put(csd_mag_workspace_bytes(L, max_order, 0));
-    w.law = put((size_t)(max_block + 1) * V * 4);
+    w.law = put((size_t)CSD_MAX_ROWS * V * 4);            // a forward may carry up to CSD_MAX_ROWS rows (catch-up chunks)
     w.qlaw = put((size_t)RING * V * 4);
     w.dl = put((size_t)(max_block > 0 ? max_block : 1) * V * 4);
     w.onehot = put((size_t)(max_block + 1) * 4);
@@ -53,7 +53,8 @@ static csd_status forward(Gen& g, int r, int from, int cnt) {
 static csd_status step(Gen& g, int r, int budget);
 
 static csd_status review(Gen& g, int r, int P, int nd) {
-    const int V = g.V, maxrows = g.max_block + 1;
+    // a forward carries as many rows as the model takes: fewer passes over the weights while catching up
+    const int V = g.V, maxrows = g.models[r]->cfg.max_rows < CSD_MAX_ROWS ? g.models[r]->cfg.max_rows : CSD_MAX_ROWS;
     int from = g.kv[r] < P - 1 ? g.kv[r] : P - 1;
     int cnt = 0;
     while (from < P + nd) {   // catch up on tokens this level has not cached, then the block itself
@@ -220,7 +221,8 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
             if (models[r]->cfg.arch == 1) rc = csd_encoder_forward(models[r], hay_dev, haystack_len, g.stream);
             for (int from = 0; rc == CSD_OK && from < init_len - 1;) {
                 int cnt = init_len - 1 - from;
-                if (cnt > max_block + 1) cnt = max_block + 1;
+                const int rows = models[r]->cfg.max_rows < CSD_MAX_ROWS ? models[r]->cfg.max_rows : CSD_MAX_ROWS;
+                if (cnt > rows) cnt = rows;
                 rc = forward(g, r, from, cnt);
                 from += cnt;
             }
