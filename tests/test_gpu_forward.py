@@ -118,3 +118,18 @@ def test_argument_and_token_errors(b):
     assert b.csd_device_status() == 6 and torch.isfinite(out).all()
     with pytest.raises(b.CsdError):
         b.Model(shape, blob[:-128])                         # blob too small
+
+
+@pytest.mark.parametrize("d_head", [32, 64, 128])
+def test_tile_edges_of_the_attention(b, orc, d_head):
+    # One layer, so that the logits follow the attention closely; block sizes chosen so that the
+    # cache length before a block, and the end of the block, fall before, on and after the 64-key
+    # tile edges and the split boundaries (1, 2, 3 ... tiles, odd remainders, a 17-row block that
+    # straddles a tile edge, a block that starts exactly on one).
+    shape = llama_shape(1, 2 * d_head, 2, 4 * d_head, 512, 600)
+    blob = workloads.make_weights(shape, seed=17, device="cuda", std=0.08, gain_std=0.2)
+    toks = workloads.make_prompt(shape.vocab, 600, seed=4)
+    blocks = [1, 17, 17, 17, 11, 1, 1, 16, 17, 14, 1, 2, 17, 17, 17, 13, 1, 5, 17, 17, 17, 17, 9, 17,
+              17, 17, 17, 17, 17, 16, 1, 3, 17, 17, 17, 17, 5]
+    assert sum(blocks) <= 600
+    run_blocks(b, orc, shape, blob, toks, blocks)
