@@ -256,8 +256,9 @@ def run_ours(args):
 
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
-            "vs_baseline": None, "dtype": "bf16 weights and K/V, fp32 accumulate", "data": "synthetic",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": WORKLOAD, "l2": "inputs (13.2 GB of weights per forward) exceed the 126 MB L2",
+                       "arithmetic": "bf16 weights and K/V, fp32 activations and accumulation",
                        "replicas": world},
             "e2e": {"value": e2e, "unit": "tokens/s", "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h},
             "gpu_launches": int(sum(s["kernel_launches"] for s in stats)),
