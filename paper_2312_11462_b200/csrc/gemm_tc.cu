@@ -34,7 +34,7 @@ int gemm_path() { return g_path; }
 static int npad_for(int m) { int c = 3 * m; return c <= 16 ? 16 : (c <= 32 ? 32 : (c <= 48 ? 48 : 64)); }
 
 struct TcPlan {
-    int npad, tiles, kblocks, grid, stages;    // kblocks: stages of work per tile (one or two 64-wide K blocks each)
+    int npad, tiles, kblocks, grid, stages, csplit;    // kblocks: stages of work per tile (one or two 64-wide K blocks each)
     size_t smem, scratch_floats;
 };
 
@@ -65,6 +65,16 @@ static TcPlan tc_plan(int m, int N, int K, bool dual) {
     if (grid < 1) grid = 1;
     if (grid > tc_sm_count()) grid = tc_sm_count();
     p.grid = (int)grid;
+    // A single-matrix GEMM with few tiles (N = 4096: 32) on a block of up to 5 rows is cut the other way:
+    // every tile goes to a cluster of four CTAs that share its K range and add their parts up through
+    // distributed shared memory, on chip, instead of parking them in global memory.  4 x 32 = 128 streaming
+    // SMs still draw the full bandwidth.  (Measured: 0.8 % faster per 7B forward at 5 rows, no gain at 9,
+    // 1 % slower at 17, hence the row limit.)
+    p.csplit = 1;
+    if (!dual && p.npad <= 16 && p.tiles * 4 <= tc_sm_count() && p.tiles * 4 >= 96 && p.kblocks >= 8) {
+        p.csplit = 4;
+        p.grid = p.tiles * 4;
+    }
     const size_t stage = (size_t)STAGE_BYTES * (dual ? 2 : ks) + (size_t)p.npad * 128 * ks;
     p.stages = (int)((TC_SMEM_MAX - 1024) / stage);
     if (p.stages > 12) p.stages = 12;
@@ -142,12 +152,13 @@ struct TcParams {
     float* Y; float* partial; unsigned* tickets; int* status;
     const float* ssq_in; int ssq_cnt;                      // rms-norm: sum of squares of the input rows, in pieces
     __nv_bfloat16* out_xs; const __nv_bfloat16* out_gain; float* out_ssq; int out_ld;
-    int N, K, ldy, nkb, tiles, stages, epilogue;
+    int N, K, ldy, nkb, tiles, stages, epilogue, csplit;
     float eps;
 };
 
 struct __align__(8) TcCtrl {
     uint64_t full[12], empty[12], acc_full[2], acc_empty[2];
+    uint64_t red_ready, red_done;      // cluster split: the leader's buffer is free / all parts have been written
     uint32_t tmem_base;
     int abort_flag, last_flag;
     float scale[32];
@@ -168,6 +179,29 @@ __device__ __forceinline__ int cta_of_unit(unsigned u, unsigned units, unsigned 
     while (c + 1 < ctas && unit_begin(c + 1, units, ctas) <= u) ++c;
     while (c > 0 && unit_begin(c, units, ctas) > u) --c;
     return (int)c;
+}
+
+// ---- distributed shared memory (cluster split) ---------------------------------------------------
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ void remote_arrive(uint32_t cluster_addr) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_addr) : "memory");
+}
+__device__ __forceinline__ void remote_store(uint32_t cluster_addr, float v) {
+    asm volatile("st.shared::cluster.f32 [%0], %1;" ::"r"(cluster_addr), "f"(v) : "memory");
+}
+__device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity) {   // acquire at cluster scope, bounded
+    const uint32_t a = smem_u32(bar);
+    for (int i = 0; i < SPIN_LIMIT; ++i) {
+        uint32_t ok;
+        asm volatile("{ .reg .pred p; mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+                     : "=r"(ok) : "r"(a), "r"(parity) : "memory");
+        if (ok) return true;
+    }
+    return false;
 }
 
 template <int M, bool DUAL>
@@ -192,12 +226,20 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int cta = blockIdx.x, ctas = gridDim.x;
     const unsigned units = (unsigned)p.tiles * (unsigned)p.nkb;
-    const unsigned u0 = unit_begin(cta, units, ctas), u1 = unit_begin(cta + 1, units, ctas);
+    unsigned u0 = unit_begin(cta, units, ctas), u1 = unit_begin(cta + 1, units, ctas);
+    const int crank = p.csplit > 1 ? cta % p.csplit : 0;     // cluster split: rank inside the tile's cluster
+    if (p.csplit > 1) {
+        const unsigned t = (unsigned)(cta / p.csplit) * (unsigned)p.nkb;
+        u0 = t + (unsigned)crank * (unsigned)p.nkb / (unsigned)p.csplit;
+        u1 = t + (unsigned)(crank + 1) * (unsigned)p.nkb / (unsigned)p.csplit;
+    }
     const int items = (int)(u1 - u0);
 
     if (tid == 0) {
         for (int s = 0; s < 12; ++s) { mbar_init(&ctl->full[s], 1); mbar_init(&ctl->empty[s], 1); }
         for (int b = 0; b < 2; ++b) { mbar_init(&ctl->acc_full[b], 1); mbar_init(&ctl->acc_empty[b], 4); }
+        mbar_init(&ctl->red_ready, 1);
+        mbar_init(&ctl->red_done, 4 * 3);               // one arrival per epilogue warp of the three other CTAs
         ctl->abort_flag = 0; ctl->last_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
@@ -211,6 +253,10 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
     tc_fence_after();
     const uint32_t tmem = ctl->tmem_base;
     volatile int* abort_flag = &ctl->abort_flag;
+    if (p.csplit > 1) {      // nobody signals a barrier of another CTA before that CTA has initialised it
+        asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+        asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+    }
     // Let the next kernel in the stream start now: its CTAs take the second slot of each SM, set
     // themselves up and request their first weight tiles while this kernel is still streaming;
     // they touch nothing this kernel writes before their own dependency wait.
@@ -343,7 +389,36 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 }
                 if (p.out_xs && p.out_gain) out_g = __bfloat162float(p.out_gain[n]);
             }
-            if (seg_len < p.nkb) {
+            if (p.csplit > 1) {
+                // Cluster split: the four CTAs of the cluster hold the four K ranges of this tile.  Rank 0
+                // finishes the tile; when its own MMAs are done its ring is free, it tells the others, they
+                // write their parts into it (distributed shared memory) and signal back, and it adds the
+                // parts in rank order.
+                constexpr int NV = NT * M;
+                float* buf = reinterpret_cast<float*>(ring);          // [3][NV][128]
+                if (crank == 0) {
+                    if (et == 0)
+                        for (int r = 1; r < p.csplit; ++r) remote_arrive(map_to_cta(smem_u32(&ctl->red_ready), (uint32_t)r));
+                    if (!mbar_wait_cluster(&ctl->red_done, 0)) *abort_flag = 1;
+#pragma unroll
+                    for (int r = 1; r < 4; ++r)
+#pragma unroll
+                        for (int u = 0; u < NT; ++u)
+#pragma unroll
+                            for (int rr = 0; rr < M; ++rr) sums[u][rr] += buf[((r - 1) * NV + u * M + rr) * TILE_N + col];
+                } else {
+                    if (!mbar_wait_cluster(&ctl->red_ready, 0)) *abort_flag = 1;
+                    const uint32_t dst = map_to_cta(smem_u32(buf), 0u);
+#pragma unroll
+                    for (int u = 0; u < NT; ++u)
+#pragma unroll
+                        for (int rr = 0; rr < M; ++rr)
+                            remote_store(dst + (uint32_t)((((crank - 1) * NV + u * M + rr) * TILE_N + col) * 4), sums[u][rr]);
+                    __syncwarp();
+                    if (lane == 0) remote_arrive(map_to_cta(smem_u32(&ctl->red_done), 0u));
+                    continue;
+                }
+            } else if (seg_len < p.nkb) {
                 // part of a tile: leave it in this CTA's slot (0 = the CTA's first segment, 1 = a later
                 // one); the CTA that arrives last adds all parts in CTA order and finishes the tile
                 float* mine = my_part + (size_t)(seg == 0 ? 0 : 1) * NT * M * TILE_N;
@@ -506,8 +581,13 @@ static csd_status launch_tc(const CUtensorMap& tw, const CUtensorMap& tw2, const
         attr_set = true;
     }
     cudaLaunchConfig_t cfg;
-    cudaLaunchAttribute attr[1];
+    cudaLaunchAttribute attr[2];
     pdl_config(cfg, attr, dim3((unsigned)pl.grid), dim3(TC_THREADS), pl.smem + 1024, st);
+    if (pl.csplit > 1) {
+        attr[1].id = cudaLaunchAttributeClusterDimension;
+        attr[1].val.clusterDim.x = (unsigned)pl.csplit; attr[1].val.clusterDim.y = 1; attr[1].val.clusterDim.z = 1;
+        cfg.numAttrs = 2;
+    }
     CSD_CUDA(cudaLaunchKernelEx(&cfg, kern, tw, tw2, tx, tp));
     count_launch();
     return CSD_OK;
@@ -540,7 +620,7 @@ csd_status launch_linear_tc(const LinearArgs& a, cudaStream_t st) {
     tp.Y = a.Y; tp.partial = a.partial; tp.tickets = a.tickets; tp.status = status_word_device();
     tp.ssq_in = a.gain ? a.ssq : nullptr; tp.ssq_cnt = ssq_cnt;
     tp.out_xs = a.out_xs; tp.out_gain = a.out_gain; tp.out_ssq = a.out_ssq; tp.out_ld = a.out_ld;
-    tp.N = a.N; tp.K = a.K; tp.ldy = a.ldy; tp.nkb = pl.kblocks; tp.tiles = pl.tiles; tp.stages = pl.stages;
+    tp.N = a.N; tp.K = a.K; tp.ldy = a.ldy; tp.nkb = pl.kblocks; tp.tiles = pl.tiles; tp.stages = pl.stages; tp.csplit = pl.csplit;
     tp.epilogue = a.epilogue; tp.eps = a.eps;
 #define CSD_TC_CASE(MM) \
     case MM: return dual ? launch_tc<MM, true>(tw, tw2, tx, tp, pl, st) : launch_tc<MM, false>(tw, tw2, tx, tp, pl, st);
