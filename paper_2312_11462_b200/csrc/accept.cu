@@ -75,6 +75,8 @@ template <bool VEC>
 __global__ void __launch_bounds__(ST_THREADS, 2)
 accept_stats_kernel(const float* __restrict__ tl, const float* __restrict__ dl, long long n_tvec, int V,
                     float invT, int greedy, StatPartial* __restrict__ out, int nchunk, long long items) {
+    pdl_wait();            // the logits come from the kernel before this one on the stream
+    pdl_trigger();
     const int lane = threadIdx.x & 31;
     const long long warps = (long long)gridDim.x * (ST_THREADS / 32);
     for (long long item = (long long)blockIdx.x * (ST_THREADS / 32) + (threadIdx.x >> 5); item < items; item += warps) {
@@ -141,6 +143,8 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
                      uint64_t seed, uint64_t step, const StatPartial* __restrict__ part, int nchunk,
                      int* __restrict__ n_acc, int* __restrict__ out_tok, RowInfo* __restrict__ info,
                      unsigned* __restrict__ tickets, int* status) {
+    pdl_wait();
+    pdl_trigger();
     const int row = blockIdx.x;
     __shared__ float s_mx[2 * MAX_K + 1];
     __shared__ float s_z[2 * MAX_K + 1];
@@ -520,12 +524,20 @@ static csd_status run_accept(const float* tl, const float* dl_in, const int32_t*
     long long ctas = (items + ST_THREADS / 32 - 1) / (ST_THREADS / 32);
     const long long cap = (long long)accept_sm_count() * 2;       // two resident CTAs per SM, grid-stride beyond
     if (ctas > cap) ctas = cap;
-    if (vec_ok)
-        accept_stats_kernel<true><<<(unsigned)ctas, ST_THREADS, 0, st>>>(tl, dl, n_tvec, V, invT, greedy, part, L.nchunk_a, items);
-    else
-        accept_stats_kernel<false><<<(unsigned)ctas, ST_THREADS, 0, st>>>(tl, dl, n_tvec, V, invT, greedy, part, L.nchunk_a, items);
-    accept_decide_kernel<<<rows, 128, 0, st>>>(tl, dl, onehot, tokens, rows, k, V, temperature, lenience, seed, step, part,
-                                               L.nchunk_a, n_acc, out_tok, info, tickets, status);
+    // both launched with programmatic stream serialisation: they are resident and waiting when their
+    // predecessor retires (in the cascade that is the output head of the review forward)
+    {
+        PdlLaunch ls(dim3((unsigned)ctas), dim3(ST_THREADS), 0, st);
+        const int greedy_i = greedy ? 1 : 0;
+        if (vec_ok)
+            CSD_CUDA(cudaLaunchKernelEx(&ls.cfg, accept_stats_kernel<true>, tl, dl, n_tvec, V, invT, greedy_i, part, L.nchunk_a, items));
+        else
+            CSD_CUDA(cudaLaunchKernelEx(&ls.cfg, accept_stats_kernel<false>, tl, dl, n_tvec, V, invT, greedy_i, part, L.nchunk_a, items));
+        PdlLaunch ld(dim3((unsigned)rows), dim3(128), 0, st);
+        CSD_CUDA(cudaLaunchKernelEx(&ld.cfg, accept_decide_kernel, tl, dl, (const int*)onehot, (const int*)tokens, rows, k, V,
+                                    temperature, lenience, seed, step, (const StatPartial*)part, L.nchunk_a, (int*)n_acc,
+                                    (int*)out_tok, info, tickets, status));
+    }
     count_launch(2);
     if (!greedy) {
         dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
