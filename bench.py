@@ -248,6 +248,20 @@ def run_ours(args):
                 "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
                 "us_per_launch": gemm_launch_us}
 
+    # every kernel class of the review step against its own HBM roofline (event pairs around each launch,
+    # so consecutive kernels do not overlap here as they do in the timed forward)
+    attn_us = 1e3 * prof["attn_ms"] / n_rev
+    accept_bytes = 4.0 * ts.vocab * (MAX_BLOCK + 1)
+    kernel_rooflines = {
+        "weight_streaming_gemm": {"bytes": weight_bytes, "us": 1e3 * prof["gemm_ms"] / n_rev, "GBps": gemm_gbs,
+                                  "frac_of_8TBps": gemm_gbs / 8000.0, "frac_of_measured": gemm_gbs / peak},
+        "block_attention": {"bytes": kv_bytes, "us": attn_us, "GBps": kv_bytes / attn_us / 1e3,
+                            "frac_of_8TBps": kv_bytes / attn_us / 1e3 / 8000.0, "note": "latency-bound at a 128-token cache"},
+        "accept": {"bytes": accept_bytes, "us": accept_us, "GBps": accept_bytes / accept_us / 1e3,
+                   "frac_of_8TBps": accept_bytes / accept_us / 1e3 / 8000.0,
+                   "note": "one row, greedy: latency-bound; the 64-row sweep is in `--configs accept`"},
+    }
+
     cpu = None
     if world == 1 and not args.no_cpu_baseline:
         n_tok, dt, _ = oracle_sample(ts, ds, tb, db, prompt, nxt)
@@ -270,7 +284,7 @@ def run_ours(args):
             "review_frac_of_measured": review_gbs / peak,
             "review_split_us": {"gemm": 1e3 * prof["gemm_ms"] / n_rev, "attention": 1e3 * prof["attn_ms"] / n_rev,
                                 "other": 1e3 * prof["other_ms"] / n_rev},
-            "accept_us": accept_us, "cascade_stats": {k: st[k] for k in ("reviews", "forwards", "drafted", "accepted",
+            "accept_us": accept_us, "kernel_rooflines": kernel_rooflines, "cascade_stats": {k: st[k] for k in ("reviews", "forwards", "drafted", "accepted",
                                                                         "mag_calls")}}
     print(json.dumps(line), flush=True)
     if world > 1:
