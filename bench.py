@@ -133,13 +133,22 @@ def run_reference(args):
     value = tokens / total
     cores = len(os.sched_getaffinity(0))
     sample = f"{ORACLE_PROMPT}-token prompt, {ORACLE_NEW} new tokens per step, same models and cascade"
+    # the oracle's own time for the two calls of a review step: one 5-row target forward over the
+    # sample's cache, and one accept call on its logits (one row, k = 4, greedy)
+    blk = prompt[ORACLE_PROMPT:ORACLE_PROMPT + MAX_BLOCK + 1]
+    t0 = time.time()
+    logits = oms[0].review_forward(blk, ORACLE_PROMPT)
+    review_s = time.time() - t0
+    t0 = time.time()
+    oracle.spec_accept(logits[None, :, :], None, np.asarray(blk[:MAX_BLOCK])[None, :], 0.0)
+    accept_s = time.time() - t0
     line = {"impl": "reference", "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": args.gpus,
             "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * total / max(len(times), 1),
             "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
             "config": {"workload": WORKLOAD, "sample": sample},
             "cpu_baseline": {"value": value, "unit": "tokens/s", "cores": cores, "kind": "oracle", "sample": sample},
             "e2e": {"value": value, "unit": "tokens/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
-            "gpu_launches": 0}
+            "gpu_launches": 0, "oracle_review_forward_s": review_s, "oracle_accept_s": accept_s}
     print(json.dumps(line), flush=True)
 
 
