@@ -207,7 +207,8 @@ int orc_spec_accept(const float* target_logits, const float* draft_logits, const
             }
             double u, u2;
             review_uniforms(seed, step, row, i, &u, &u2);
-            double lhs = u * qx, rhs = l * p[x];
+            /* Appendix B: no lenience between the statistical drafter and its reviewer */
+            double lhs = u * qx, rhs = (point_mass ? 1.0 : l) * p[x];
             double big = lhs > rhs ? lhs : rhs;
             if (fabs(lhs - rhs) <= 1e-5 * big) flag |= 1;
             if (lhs < rhs) continue; /* accepted */

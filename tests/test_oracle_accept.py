@@ -226,3 +226,25 @@ def test_bad_arguments(orc):
         orc.spec_accept(t, None, np.zeros((1, 1)), 1.0, lenience=0.5)
     with pytest.raises(ValueError):
         orc.spec_accept(t, None, np.zeros((1, 1)), -1.0)
+
+
+def test_no_lenience_for_point_mass_positions(orc):
+    # Appendix B: lenience is not used between the statistical drafter and its reviewer
+    V, N, x = 8, 50_000, 2
+    t, d = workloads.small_logits(1, 2, V, seed=23, scale=1.5)
+    tl = np.broadcast_to(t[0], (N, 3, V))
+    dl = np.broadcast_to(d[0], (N, 2, V))
+    tok = np.broadcast_to(np.array([x, x]), (N, 2))
+    # all point mass: any lenience gives the very same outcome as lenience 1
+    a = orc.spec_accept(tl, None, tok, 1.0, lenience=1.0, seed=3)
+    b = orc.spec_accept(tl, None, tok, 1.0, lenience=7.0, seed=3)
+    assert (a[0] == b[0]).all() and (a[1] == b[1]).all()
+    # mixed block: position 0 carries a law (lenience applies), position 1 is a point mass (it does not)
+    p, q = softmax(t[0]), softmax(d[0])
+    oh = np.broadcast_to(np.array([0, 1]), (N, 2))
+    l = 3.0
+    n, _, _ = orc.spec_accept(tl, dl, tok, 1.0, lenience=l, seed=4, onehot=oh)
+    a0 = min(1.0, l * p[0][x] / q[0][x])        # P(position 0 accepted | x drawn) under lenience
+    a1 = p[1][x]                                 # point mass: accepted with probability p(x), no lenience
+    assert abs((n >= 1).mean() - a0) < 4 * np.sqrt(a0 * (1 - a0) / N + 1e-12) + 1e-9
+    assert abs((n == 2).mean() - a0 * a1) < 4 * np.sqrt(a0 * a1 * (1 - a0 * a1) / N)
