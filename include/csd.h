@@ -162,7 +162,9 @@ csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, 
  *   temperature == 0: greedy review: x_i is accepted iff it is the argmax of target_logits[i]
  *     (ties: smallest index); the output token is the argmax at the first mismatch (or at k).
  * q_i is softmax(draft_logits[i] / T), or the point mass on x_i where draft_logits_dev is NULL
- * or onehot_dev[row, i] != 0 (statistical drafter).
+ * or onehot_dev[row, i] != 0 (statistical drafter).  Lenience multiplies p_i only at positions
+ * whose proposal carries a law; a point-mass position is tested with lenience 1 (Appendix B: no
+ * lenience between the statistical drafter and its reviewer).
  * Uniforms: Philox4x32-10 with key (seed lo, seed hi) and counter (i, row, step lo, step hi);
  * word 0 -> u_i, word 1 -> the resampling uniform of position i; u = (word >> 8) * 2^-24.  The
  * resample is the inverse CDF in vocabulary order (smallest j with cumulative mass > u * total),

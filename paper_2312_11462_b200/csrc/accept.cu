@@ -208,7 +208,7 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
             if (!point)
                 qx = exp(((double)dl[((long long)row * k + i) * V + x] - (double)s_mx[k + 1 + i]) / T) /
                      (double)s_z[k + 1 + i];
-            accept = u * qx < (double)lenience * px;
+            accept = u * qx < (point ? 1.0 : (double)lenience) * px;   // no lenience for the statistical drafter's tokens (Appendix B)
         }
         s_acc[i] = accept ? 1 : 0; s_x[i] = x; s_point[i] = point ? 1 : 0; s_u2[i] = word_uniform(r.w[1]);
     }

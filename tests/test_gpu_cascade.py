@@ -112,20 +112,26 @@ def test_teacher_forced_logits_follow_the_oracle(b, orc):
 
 @pytest.mark.parametrize("lenience", [1.0, 3.0])
 def test_sampling_cascade_matches_oracle_decisions(b, orc, lenience):
-    # same Philox stream, same laws => same accepted counts and tokens while logits agree
-    # (lenience > 1, Section 3.1, loosens the accept test where the draft reviews Max-Gram tokens)
+    # same Philox stream, same laws => same accepted counts and tokens while logits agree.
+    # With lenience > 1 (Section 3.1) a second neural draft sits below the first, so that a draft
+    # reviews a draft's tokens, the one place where lenience applies (Appendix B).
     ts, ds = SHAPES["tiny_target"], SHAPES["tiny_draft"]
-    tb = workloads.make_weights(ts, seed=0, device="cuda", std=0.05)
-    db = workloads.make_weights(ds, seed=1, device="cuda", std=0.05)
+    blobs = [workloads.make_weights(ts, seed=0, device="cuda", std=0.05),
+             workloads.make_weights(ds, seed=1, device="cuda", std=0.05)]
+    shapes = [ts, ds]
+    K = [[2, 2], [0, 3]]
+    if lenience > 1.0:
+        blobs.append(workloads.make_weights(ds, seed=2, device="cuda", std=0.05))
+        shapes.append(ds)
+        K = [[2, 1, 1], [0, 2, 2], [0, 0, 3]]
     prompt = workloads.make_repetitive_prompt(ts.vocab, 32, seed=5)
     nxt = workloads.bigram_table(prompt, ts.vocab, seed=0)
-    K = [[2, 2], [0, 3]]
     agree = 0
     for seed in range(6):
-        oms = [orc.Model(ts, orc.blob_to_u16(tb)), orc.Model(ds, orc.blob_to_u16(db))]
+        oms = [orc.Model(sh, orc.blob_to_u16(w)) for sh, w in zip(shapes, blobs)]
         want, _, _ = orc.cascade_generate(oms, prompt, nxt, K, 4, prompt, 24, temperature=1.0, lenience=lenience,
                                            seed=seed)
-        gms = [b.Model(ts, tb), b.Model(ds, db)]
+        gms = [b.Model(sh, w) for sh, w in zip(shapes, blobs)]
         got, st = b.Cascade(gms, K, 4, to_dev_i32(nxt), 64).csd_cascade_generate(prompt, prompt, 24, 1.0, lenience, seed)
         assert len(got) == 24 and ((got >= 0) & (got < ts.vocab)).all()
         agree += int(np.array_equal(got, want))
