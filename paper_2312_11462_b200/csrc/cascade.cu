@@ -37,7 +37,7 @@ struct Gen {
     uint64_t seed, step = 0; csd_mag* mag = nullptr; int V, cap;
     int32_t* seq; int len = 0; int kv[8] = {0};
     std::vector<signed char> src;        // per position: proposing level, -1 = point mass
-    float *law, *qlaw, *dl; int32_t *onehot_dev, *result_dev; void* accept_ws; size_t accept_bytes;
+    float *law, *qlaw, *dl; int32_t *onehot_dev, *result_dev, *result_map = nullptr; void* accept_ws; size_t accept_bytes;
     int32_t* pinned = nullptr;           // [0..1] = (n_acc, out_tok); [2..] = onehot flags staging
     csd_cascade_stats* st; cudaStream_t stream;
     cudaEvent_t ev_decode; bool decode_marked = false;
@@ -87,13 +87,14 @@ static csd_status review(Gen& g, int r, int P, int nd) {
     }
     const float len_r = r == 0 ? 1.f : g.lenience;   // lenience never applies when the target reviews
     csd_status s = csd_spec_accept(target, dl, onehot, g.seq + P, 1, nd, V, g.temperature, len_r, g.seed, g.step++,
-                                   g.result_dev, g.result_dev + 1, g.accept_ws, g.accept_bytes, g.stream);
+                                   g.result_map, g.result_map + 1, g.accept_ws, g.accept_bytes, g.stream);
     if (s != CSD_OK) return s;
-    CSD_CUDA(cudaMemcpyAsync(g.pinned, g.result_dev, 8, cudaMemcpyDeviceToHost, g.stream));
+    // the accept kernels write (n_acc, out token) straight into mapped pinned host memory: no copy to wait for
     CSD_CUDA(cudaStreamSynchronize(g.stream));
     const int n_acc = g.pinned[0];
     if (n_acc < 0 || n_acc > nd) return CSD_ERR_CUDA;
-    CSD_CUDA(cudaMemcpyAsync(g.seq + P + n_acc, g.result_dev + 1, 4, cudaMemcpyDeviceToDevice, g.stream));
+    g.pinned[CSD_MAX_ROWS + 8] = g.pinned[1];     // (a slot the next review does not overwrite while this copy is in flight)
+    CSD_CUDA(cudaMemcpyAsync(g.seq + P + n_acc, g.pinned + CSD_MAX_ROWS + 8, 4, cudaMemcpyHostToDevice, g.stream));
     g.st->reviews[r] += 1;
     g.st->drafted[r] += nd;
     g.st->accepted[r] += n_acc;
@@ -200,7 +201,11 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
     g.accept_ws = ws + w.accept; g.accept_bytes = w.total - w.accept;
     g.src.assign((size_t)g.cap + 64, 0);
 
-    CSD_CUDA(cudaHostAlloc((void**)&g.pinned, (size_t)(2 + CSD_MAX_ROWS + 64) * 4, cudaHostAllocDefault));
+    CSD_CUDA(cudaHostAlloc((void**)&g.pinned, (size_t)(2 + CSD_MAX_ROWS + 64) * 4, cudaHostAllocMapped));
+    if (cudaHostGetDevicePointer((void**)&g.result_map, g.pinned, 0) != cudaSuccess || !g.result_map) {
+        cudaFreeHost(g.pinned);
+        return note_cuda(cudaGetLastError());
+    }
     cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
     csd_status rc = CSD_OK;
     auto fail = [&](csd_status s) { rc = s; };
