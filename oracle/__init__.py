@@ -37,13 +37,13 @@ class ModelConfig(C.Structure):
 class Stats(C.Structure):
     _fields_ = [("tokens", C.c_int64), ("reviews", C.c_int64 * 8), ("forwards", C.c_int64 * 8),
                 ("drafted", C.c_int64 * 8), ("accepted", C.c_int64 * 8), ("mag_calls", C.c_int64),
-                ("mag_tokens", C.c_int64)]
+                ("mag_tokens", C.c_int64), ("near_ties", C.c_int64), ("first_near_tie", C.c_int64)]
 
     def as_dict(self, n_levels: int):
         return dict(tokens=self.tokens, reviews=list(self.reviews)[:n_levels],
                     forwards=list(self.forwards)[:n_levels], drafted=list(self.drafted)[:n_levels],
                     accepted=list(self.accepted)[:n_levels], mag_calls=self.mag_calls,
-                    mag_tokens=self.mag_tokens)
+                    mag_tokens=self.mag_tokens, near_ties=self.near_ties, first_near_tie=self.first_near_tie)
 
 
 def lib():
@@ -56,6 +56,9 @@ def lib():
         L.orc_double_to_bf16.argtypes = [C.c_double]
         L.orc_double_to_bf16.restype = C.c_uint16
         L.orc_set_kv_exact.argtypes = [C.c_int]
+        L.orc_set_linear_f32.argtypes = [C.c_int]
+        L.orc_top2_margin.argtypes = [C.c_void_p, C.c_int]
+        L.orc_top2_margin.restype = C.c_float
         L.orc_spec_accept.argtypes = [C.c_void_p, C.c_void_p, C.c_void_p, C.c_void_p, C.c_int, C.c_int,
                                       C.c_int, C.c_float, C.c_float, C.c_uint64, C.c_uint64,
                                       C.c_void_p, C.c_void_p, C.c_void_p]
@@ -72,7 +75,7 @@ def lib():
         L.orc_review_forward.argtypes = [C.c_void_p, C.c_void_p, C.c_int, C.c_int, C.c_void_p]
         L.orc_cascade_generate.argtypes = [C.c_void_p, C.c_int, C.c_void_p, C.c_int, C.c_void_p, C.c_int,
                                            C.c_void_p, C.c_int, C.c_float, C.c_float, C.c_uint64,
-                                           C.c_void_p, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
+                                           C.c_void_p, C.c_int, C.c_int, C.c_int, C.c_void_p, C.c_void_p,
                                            C.c_void_p, C.c_void_p]
     return _lib
 
@@ -111,6 +114,16 @@ def double_to_bf16(x: float) -> int:
 def set_kv_exact(on: bool) -> None:
     """Test hook: keep cached K/V unrounded (for comparison with library models)."""
     lib().orc_set_kv_exact(int(on))
+
+
+def set_linear_f32(on: bool) -> None:
+    """Test hook: round every contraction result to fp32 (a second correct way to do the sums)."""
+    lib().orc_set_linear_f32(int(on))
+
+
+def top2_margin(logits) -> float:
+    x = _f32(logits).ravel()
+    return float(lib().orc_top2_margin(_p(x), len(x)))
 
 
 def spec_accept(target_logits, draft_logits, tokens, temperature: float, lenience: float = 1.0,
@@ -212,7 +225,7 @@ def blob_to_u16(blob) -> np.ndarray:
 
 def cascade_generate(models: Sequence[Model], haystack, bigram_next, K, max_block: int,
                      init_seq, max_new: int, temperature: float = 0.0, lenience: float = 1.0,
-                     seed: int = 0, max_order: int = 16):
+                     seed: int = 0, max_order: int = 16, dynamic_haystack: bool = False):
     """Returns (tokens, margins, stats dict).  models[0] is the target."""
     n = len(models)
     arr = (C.c_void_p * n)(*[m.h for m in models])
@@ -226,7 +239,7 @@ def cascade_generate(models: Sequence[Model], haystack, bigram_next, K, max_bloc
     st = Stats()
     rc = lib().orc_cascade_generate(arr, n, _p(hay), len(hay), _p(big), max_order, _p(Km), max_block,
                                     lenience, temperature, seed, _p(init), len(init), max_new,
-                                    _p(out), C.byref(out_len), _p(margins), C.byref(st))
+                                    int(dynamic_haystack), _p(out), C.byref(out_len), _p(margins), C.byref(st))
     if rc:
         raise ValueError(f"orc_cascade_generate failed ({rc})")
     return out[:out_len.value].copy(), margins[:out_len.value].copy(), st.as_dict(n)

@@ -11,9 +11,9 @@
  *
  * What each part follows:
  *   orc_spec_accept      Section 2 (proposing / reviewing stages), Section 3.1 (lenience, greedy)
- *   orc_mag_draft        Section 3.3 and the Max-Gram listing of Appendix A
- *   orc_review_forward   "reviewed by a target model in parallel ... in one single run"
- *                        (Section 1); the architectures are the families named in Section 5.1
+ *   orc_mag_draft        Section 3.3 (the definition in words; Appendix A gives a tensor formulation)
+ *   orc_review_forward   the reviewer scores every drafted position in ONE forward pass
+ *                        (Sections 1 and 2); the architectures are the families named in Section 5.1
  *   orc_cascade_generate Algorithm 1 (for-loop = horizontal cascade, recursion = vertical)
  *   orc_philox4x32_10    Salmon et al., "Parallel random numbers: as easy as 1, 2, 3" (SC'11)
  *
@@ -242,39 +242,22 @@ int orc_spec_accept(const float* target_logits, const float* draft_logits, const
 /* Max-Gram (Section 3.3, Appendix A)                                                         */
 /* ------------------------------------------------------------------------------------------ */
 /*
- * One search, in the listing's steps: mark the haystack positions equal to the last token,
- * then for i = 2, 3, ... keep the i-gram starts whose first token equals the i-th token from
- * the end; when no i-gram survives, the FIRST surviving (i-1)-gram decides.  A candidate must
- * be followed by at least one haystack token (so the proposal is never empty, and a sequence
- * that still ends with the haystack itself does not match its own tail).  `max_order` caps i.
- * Returns the haystack index of the token after the match, or -1 without any match.
+ * One search, as Section 3.3 words it: the longest run of tokens at the end of the sequence (at
+ * most max_order of them) that also occurs in the haystack, the earliest such occurrence.  An
+ * occurrence counts only if at least one haystack token follows it (so the proposal is never
+ * empty, and a sequence that still ends with the haystack itself does not match its own tail).
+ * Returns the haystack index of the token after the occurrence, or -1 without any match.
  */
-static int mag_search(const int32_t* hay, int L, const int32_t* seq, int T, int max_order,
-                      uint8_t* matches, uint8_t* combined) {
-    if (T < 1 || L < 2) return -1;
-    int any = 0;
-    /* matches[j] = 1 iff a 1-gram match sits at j and j+1 < L */
-    for (int j = 0; j < L; ++j) {
-        matches[j] = (uint8_t)(j + 1 < L && hay[j] == seq[T - 1]);
-        any |= matches[j];
-    }
-    if (!any) return -1;
-    int order = 1; /* matches[] holds the starts of `order`-gram matches */
-    int limit = T < max_order ? T : max_order;
-    for (int i = 2; i <= limit; ++i) {
-        int n_starts = L - (i - 1); /* possible starts of an i-gram */
-        int any_i = 0;
-        for (int j = 0; j < n_starts; ++j) {
-            combined[j] = (uint8_t)(hay[j] == seq[T - i] && matches[j + 1]);
-            any_i |= combined[j];
+static int mag_search(const int32_t* hay, int L, const int32_t* seq, int T, int max_order) {
+    int longest = T < max_order ? T : max_order;
+    for (int order = longest; order >= 1; --order) {
+        const int32_t* tail = seq + (T - order);
+        for (int j = 0; j + order < L; ++j) {
+            int same = 1;
+            for (int e = 0; e < order && same; ++e) same = hay[j + e] == tail[e];
+            if (same) return j + order;
         }
-        if (!any_i) break;
-        memcpy(matches, combined, (size_t)n_starts);
-        for (int j = n_starts; j < L; ++j) matches[j] = 0;
-        order = i;
     }
-    for (int j = 0; j < L; ++j)
-        if (matches[j]) return j + order;
     return -1;
 }
 
@@ -287,12 +270,10 @@ int orc_mag_draft(const int32_t* hay, int L, const int32_t* bigram_next, int V, 
                   int T, int n, int max_order, int32_t* out) {
     if (T < 1 || n < 0 || max_order < 1) return -1;
     int32_t* cur = (int32_t*)malloc(sizeof(int32_t) * (size_t)(T + n));
-    uint8_t* m1 = (uint8_t*)malloc((size_t)(L > 0 ? L : 1));
-    uint8_t* m2 = (uint8_t*)malloc((size_t)(L > 0 ? L : 1));
     memcpy(cur, seq, sizeof(int32_t) * (size_t)T);
     int len = T, made = 0;
     while (made < n) {
-        int idx = mag_search(hay, L, cur, len, max_order, m1, m2);
+        int idx = mag_search(hay, L, cur, len, max_order);
         if (idx < 0) {
             int32_t last = cur[len - 1];
             int32_t nx = (last >= 0 && last < V) ? bigram_next[last] : 0;
@@ -305,7 +286,7 @@ int orc_mag_draft(const int32_t* hay, int L, const int32_t* bigram_next, int V, 
             }
         }
     }
-    free(cur); free(m1); free(m2);
+    free(cur);
     return made;
 }
 
@@ -428,6 +409,12 @@ void orc_model_destroy(orc_model* m) {
     free(m);
 }
 
+/* Test hook: with `on`, every result of a contraction is rounded to fp32 before it is used.  That
+   is a second, equally correct way to carry the arithmetic; the tests use it to measure how far two
+   correct implementations drift apart once both round K/V to bf16. */
+static int g_linear_f32 = 0;
+void orc_set_linear_f32(int on) { g_linear_f32 = on; }
+
 /* Y[r][n] = sum_k X[r][k] * W[n][k]; W bf16 [N,K] row-major */
 static void linear(const uint16_t* W, int N, int K, const double* X, int m, double* Y) {
 #pragma omp parallel for schedule(static)
@@ -437,7 +424,7 @@ static void linear(const uint16_t* W, int N, int K, const double* X, int m, doub
             const double* x = X + (size_t)r * K;
             double acc = 0.0;
             for (int k = 0; k < K; ++k) acc += bf16_to_double(w[k]) * x[k];
-            Y[(size_t)r * N + n] = acc;
+            Y[(size_t)r * N + n] = g_linear_f32 ? (double)(float)acc : acc;
         }
     }
 }
@@ -617,9 +604,9 @@ int orc_encoder_forward(orc_model* M, const int32_t* tokens, int n) {
  * last committed token).  Reads cache rows [0, kv_len), writes rows [kv_len, kv_len+m), and
  * returns fp32 logits [m, V]; row r is the model's next-token law after position kv_len+r.
  */
-int orc_review_forward(orc_model* M, const int32_t* tokens, int m, int kv_len, float* logits) {
+static int forward_rows(orc_model* M, const int32_t* tokens, int m, int kv_len, float* logits, int first_row) {
     const orc_model_config* c = &M->c;
-    if (m < 1 || kv_len < 0 || kv_len + m > c->max_seq) return 1;
+    if (m < 1 || kv_len < 0 || kv_len + m > c->max_seq || first_row < 0 || first_row >= m) return 1;
     if (c->arch == 1 && M->enc_len < 1) return 2;
     int d = c->d_model, H = c->n_heads, Dh = c->d_head, di = H * Dh, ff = c->d_ff, V = c->vocab;
     double* x = (double*)malloc(sizeof(double) * (size_t)m * d);
@@ -631,7 +618,8 @@ int orc_review_forward(orc_model* M, const int32_t* tokens, int m, int kv_len, f
     double* tmp = (double*)malloc(sizeof(double) * (size_t)m * d);
     double* g = (double*)malloc(sizeof(double) * (size_t)m * ff);
     double* u = (double*)malloc(sizeof(double) * (size_t)m * ff);
-    double* lg = (double*)malloc(sizeof(double) * (size_t)m * V);
+    int n_out = m - first_row;      /* logits are wanted for rows first_row .. m-1 */
+    double* lg = (double*)malloc(sizeof(double) * (size_t)n_out * V);
     for (int r = 0; r < m; ++r) {
         int t = tokens[r];
         if (t < 0 || t >= V) t = 0;
@@ -700,48 +688,57 @@ int orc_review_forward(orc_model* M, const int32_t* tokens, int m, int kv_len, f
         ffn_block(M, y, x, m, h, g, u, tmp);
     }
     for (int r = 0; r < m; ++r) rmsnorm(x + (size_t)r * d, M->final_norm, d, c->norm_eps, h + (size_t)r * d);
-    linear(M->lm_head, V, d, h, m, lg);
-    for (size_t i = 0; i < (size_t)m * V; ++i) logits[i] = (float)lg[i];
+    linear(M->lm_head, V, d, h + (size_t)first_row * d, n_out, lg);
+    for (size_t i = 0; i < (size_t)n_out * V; ++i) logits[i] = (float)lg[i];
     free(x); free(h); free(q); free(k); free(v); free(o); free(tmp); free(g); free(u); free(lg);
     return 0;
+}
+
+int orc_review_forward(orc_model* M, const int32_t* tokens, int m, int kv_len, float* logits) {
+    return forward_rows(M, tokens, m, kv_len, logits, 0);
 }
 
 /* ------------------------------------------------------------------------------------------ */
 /* Algorithm 1: CascadeSpeculativeDraftingStep, driven until max_new tokens exist             */
 /* ------------------------------------------------------------------------------------------ */
+/*
+ * Written for checking by eye, not for speed: nothing is cached between reviews.  A review runs
+ * the reviewing model over the WHOLE sequence with a fresh cache and keeps the rows it needs, and
+ * the law every pending token was drawn from is kept in a plain per-position list (curProbs of
+ * the algorithm).  The result does not depend on this choice: a position's K/V and logits are
+ * functions of the tokens before it alone.
+ */
 typedef struct {
     int64_t tokens;             /* tokens generated */
     int64_t reviews[8];         /* review calls per level (0 = target) */
-    int64_t forwards[8];        /* forward passes per level, catch-up chunks included */
+    int64_t forwards[8];        /* forward passes per level (one per review here) */
     int64_t drafted[8];         /* drafted tokens presented to the level's reviews */
     int64_t accepted[8];        /* of which accepted */
     int64_t mag_calls;
     int64_t mag_tokens;
+    int64_t near_ties;          /* reviews whose decision lay within rounding of a threshold */
+    int64_t first_near_tie;     /* index (among generated tokens) where the first such review began, -1: none */
 } orc_stats;
 
 typedef struct {
-    int n_levels;               /* neural models: level 0 = target, 1.. = drafts */
+    int n_levels;               /* neural models: level 0 = target, 1.. = drafts; level n_levels = Max-Gram */
     orc_model** models;
     const int32_t* hay; int L;  /* Max-Gram haystack */
+    int dynamic_hay;            /* 1: the haystack is followed by everything generated so far */
     const int32_t* bigram; int max_order;
-    const int32_t* K; int n;    /* n x n budget matrix, n = n_levels (neural drafts + Max-Gram) */
+    const int32_t* K;           /* n_levels x n_levels budget matrix */
     int max_block;              /* most drafted tokens one review takes */
     double lenience; float temperature;
     uint64_t seed, step;
-    int32_t* seq; int len;      /* current sequence */
-    int* kv;                    /* per level: number of leading tokens whose K/V are cached */
-    int* src;                   /* per position: level whose law proposed the token, -1 = point mass */
-    float* qlaw;                /* ring of proposing laws (fp32 logits), row = position % RING */
-    float* law;                 /* scratch: the reviewer's logits, (max_block+1) rows */
-    int V, cap;
+    int32_t* seq; int len;      /* curGen */
+    float** probs;              /* curProbs: per position the fp32 logits of the law that proposed the
+                                   token, NULL = point mass (prefix and Max-Gram tokens) */
+    int V, cap, init_len;
     float* margins;             /* optional: top-2 logit margin of the target at each new token */
-    int prefix_len;
     orc_stats* st;
 } cascade;
 
-#define RING 128
-
-static float top2_margin(const float* x, int V) {
+float orc_top2_margin(const float* x, int V) {
     float a = -INFINITY, b = -INFINITY;
     for (int j = 0; j < V; ++j) {
         if (x[j] > a) { b = a; a = x[j]; }
@@ -750,85 +747,99 @@ static float top2_margin(const float* x, int V) {
     return a - b;
 }
 
-/* Appends `budget` Max-Gram tokens (r == n_levels) or runs one drafting+review step of neural
-   level r.  New tokens land in cs->seq with their proposing law recorded. */
-static int cascade_step(cascade* cs, int r, int budget) {
-    if (r == cs->n_levels) { /* base case: the statistical drafter generates directly */
-        if (budget < 1) budget = 1;
-        if (cs->len + budget > cs->cap) return 3;
-        orc_mag_draft(cs->hay, cs->L, cs->bigram, cs->V, cs->seq, cs->len, budget, cs->max_order,
-                      cs->seq + cs->len);
-        for (int i = 0; i < budget; ++i) cs->src[cs->len + i] = -1;
-        cs->len += budget;
-        cs->st->mag_calls += 1;
-        cs->st->mag_tokens += budget;
-        return 0;
+static void set_prob(cascade* cs, int pos, const float* logits) {
+    free(cs->probs[pos]);
+    cs->probs[pos] = NULL;
+    if (logits) {
+        cs->probs[pos] = (float*)malloc(sizeof(float) * (size_t)cs->V);
+        memcpy(cs->probs[pos], logits, sizeof(float) * (size_t)cs->V);
     }
-    int P = cs->len;
-    /* horizontal cascade: slot c of row r of K is drafted by level c+1 */
-    for (int c = r; c < cs->n; ++c) {
-        int kc = cs->K[(size_t)r * cs->n + c];
-        if (kc <= 0) continue;
-        int start = cs->len;
-        while (cs->len - start < kc) {
-            int rc = cascade_step(cs, c + 1, kc - (cs->len - start)); /* vertical cascade */
-            if (rc) return rc;
-        }
+}
+
+/* The statistical drafter appends `want` tokens (base case of the recursion). */
+static int statistical_draft(cascade* cs, int want) {
+    if (want < 1) want = 1;
+    if (cs->len + want > cs->cap) return 3;
+    const int32_t* hay = cs->hay;
+    int L = cs->L;
+    int32_t* joined = NULL;
+    if (cs->dynamic_hay) {      /* Section 3.3: "... the initial input (or existing generation)": both */
+        int gen = cs->len - cs->init_len;
+        joined = (int32_t*)malloc(sizeof(int32_t) * (size_t)(L + gen + 1));
+        memcpy(joined, cs->hay, sizeof(int32_t) * (size_t)L);
+        memcpy(joined + L, cs->seq + cs->init_len, sizeof(int32_t) * (size_t)gen);
+        hay = joined;
+        L += gen;
     }
-    int nd = cs->len - P;
-    if (nd > cs->max_block) nd = cs->max_block; /* surplus drafts are dropped before the review */
-    cs->len = P + nd;
-    if (P + nd + 1 > cs->cap) return 3;
-    /* review by level r: forward over every token it has not cached yet; the last call covers
-       inputs P-1 .. P+nd-1, whose output rows are the laws of positions P .. P+nd */
-    orc_model* M = cs->models[r];
-    int V = cs->V, maxrows = cs->max_block + 1;
-    int from = cs->kv[r];
-    if (from > P - 1) from = P - 1;
-    while (from < P + nd) {
-        int cnt = P + nd - from;
-        if (cnt > maxrows) cnt = (from + maxrows <= P - 1) ? maxrows : (P - 1) - from;
-        float* tmp = (float*)malloc(sizeof(float) * (size_t)cnt * V);
-        if (orc_review_forward(M, cs->seq + from, cnt, from, tmp)) { free(tmp); return 4; }
-        for (int i = 0; i < cnt; ++i) { /* row i is the law of position from+i+1 */
-            int pos = from + i + 1;
-            if (pos >= P) memcpy(cs->law + (size_t)(pos - P) * V, tmp + (size_t)i * V, sizeof(float) * (size_t)V);
-        }
-        free(tmp);
-        from += cnt;
-        cs->st->forwards[r] += 1;
-    }
-    /* gather the proposing laws of the drafted tokens */
+    orc_mag_draft(hay, L, cs->bigram, cs->V, cs->seq, cs->len, want, cs->max_order, cs->seq + cs->len);
+    free(joined);
+    for (int i = 0; i < want; ++i) set_prob(cs, cs->len + i, NULL);
+    cs->len += want;
+    cs->st->mag_calls += 1;
+    cs->st->mag_tokens += want;
+    return 0;
+}
+
+/* review(M, curGen, curProbs, l) of Algorithm 1 for the nd pending tokens at positions P .. P+nd-1 */
+static int review(cascade* cs, int r, int P, int nd) {
+    int V = cs->V;
+    float* law = (float*)malloc(sizeof(float) * (size_t)(nd + 1) * V);
+    /* inputs 0 .. P+nd-1; output row j is the law of position j+1, so rows P-1 .. P+nd-1 are wanted */
+    if (forward_rows(cs->models[r], cs->seq, P + nd, 0, law, P - 1)) { free(law); return 4; }
+    cs->st->forwards[r] += 1;
     float* dl = NULL;
     int32_t* onehot = (int32_t*)calloc((size_t)(nd > 0 ? nd : 1), sizeof(int32_t));
     if (cs->temperature > 0.0f && nd > 0) {
         dl = (float*)calloc((size_t)nd * V, sizeof(float));
         for (int i = 0; i < nd; ++i) {
-            if (cs->src[P + i] < 0) onehot[i] = 1;
-            else memcpy(dl + (size_t)i * V, cs->qlaw + (size_t)((P + i) % RING) * V, sizeof(float) * (size_t)V);
+            if (!cs->probs[P + i]) onehot[i] = 1;
+            else memcpy(dl + (size_t)i * V, cs->probs[P + i], sizeof(float) * (size_t)V);
         }
     }
-    int32_t n_acc = 0, out_tok = 0;
-    float len_r = (r == 0) ? 1.0f : (float)cs->lenience; /* no lenience when the target reviews */
-    orc_spec_accept(cs->law, dl, onehot, cs->seq + P, 1, nd, V, cs->temperature, len_r, cs->seed,
-                    cs->step++, &n_acc, &out_tok, NULL);
+    int32_t n_acc = 0, out_tok = 0, tie = 0;
+    float l = (r == 0) ? 1.0f : (float)cs->lenience;   /* "if isFirstCall: l <- 1" */
+    orc_spec_accept(law, dl, onehot, cs->seq + P, 1, nd, V, cs->temperature, l, cs->seed, cs->step++,
+                    &n_acc, &out_tok, &tie);
     free(dl); free(onehot);
+    if (tie) {
+        if (cs->st->near_ties == 0) cs->st->first_near_tie = P - cs->init_len;
+        cs->st->near_ties += 1;
+    }
     cs->st->reviews[r] += 1;
     cs->st->drafted[r] += nd;
     cs->st->accepted[r] += n_acc;
-    cs->len = P + n_acc;
-    cs->seq[cs->len] = out_tok;
-    /* tokens P .. P+n_acc now follow level r's own law (rows 0 .. n_acc of its logits) */
+    /* the accepted tokens and the one emitted after them now follow level r's own law */
+    cs->seq[P + n_acc] = out_tok;
     for (int i = 0; i <= n_acc; ++i) {
-        cs->src[P + i] = r;
-        if (r > 0) memcpy(cs->qlaw + (size_t)((P + i) % RING) * V, cs->law + (size_t)i * V, sizeof(float) * (size_t)V);
-        if (r == 0 && cs->margins) cs->margins[P + i - cs->prefix_len] = top2_margin(cs->law + (size_t)i * V, V);
+        set_prob(cs, P + i, r > 0 ? law + (size_t)i * V : NULL);
+        if (r == 0 && cs->margins) cs->margins[P + i - cs->init_len] = orc_top2_margin(law + (size_t)i * V, V);
     }
-    cs->len += 1;
-    cs->kv[r] = P + n_acc;
-    for (int c = r + 1; c < cs->n_levels; ++c)
-        if (cs->kv[c] > P + n_acc) cs->kv[c] = P + n_acc;
+    for (int i = n_acc + 1; i < nd; ++i) set_prob(cs, P + i, NULL);   /* rejected tokens are gone */
+    cs->len = P + n_acc + 1;
+    free(law);
     return 0;
+}
+
+/* One call of the algorithm with level r as the reviewer ("target" of the call) and the levels
+   below it as its draft list; r == n_levels is the call whose draft list is empty. */
+static int cascade_step(cascade* cs, int r, int want) {
+    if (r == cs->n_levels) return statistical_draft(cs, want);
+    int n = cs->n_levels, P = cs->len;
+    for (int i = r; i < n; ++i) {                 /* horizontal cascade: slot i belongs to level i + 1 */
+        int k_i = cs->K[(size_t)r * n + i];
+        if (k_i <= 0) continue;
+        int slot_start = cs->len;
+        while (cs->len - slot_start < k_i) {      /* vertical cascade */
+            int rc = cascade_step(cs, i + 1, k_i - (cs->len - slot_start));
+            if (rc) return rc;
+        }
+    }
+    int nd = cs->len - P;
+    for (int i = cs->max_block; i < nd; ++i) set_prob(cs, P + i, NULL);   /* surplus drafts are dropped */
+    if (nd > cs->max_block) nd = cs->max_block;
+    cs->len = P + nd;
+    if (P + nd + 1 > cs->cap) return 3;
+    return review(cs, r, P, nd);
 }
 
 /*
@@ -841,37 +852,36 @@ static int cascade_step(cascade* cs, int r, int budget) {
 int orc_cascade_generate(orc_model** models, int n_levels, const int32_t* hay, int L,
                          const int32_t* bigram_next, int max_order, const int32_t* K,
                          int max_block, float lenience, float temperature, uint64_t seed,
-                         const int32_t* init_seq, int init_len, int max_new, int32_t* out_tokens,
-                         int32_t* out_len, float* margins, orc_stats* stats) {
+                         const int32_t* init_seq, int init_len, int max_new, int dynamic_hay,
+                         int32_t* out_tokens, int32_t* out_len, float* margins, orc_stats* stats) {
     if (n_levels < 1 || n_levels > 7 || init_len < 1 || max_new < 0 || max_block < 0) return 1;
     cascade cs;
     memset(&cs, 0, sizeof(cs));
     orc_stats local;
     cs.st = stats ? stats : &local;
     memset(cs.st, 0, sizeof(orc_stats));
+    cs.st->first_near_tie = -1;
     cs.n_levels = n_levels; cs.models = models;
-    cs.hay = hay; cs.L = L; cs.bigram = bigram_next; cs.max_order = max_order;
-    cs.K = K; cs.n = n_levels; cs.max_block = max_block;
+    cs.hay = hay; cs.L = L; cs.dynamic_hay = dynamic_hay; cs.bigram = bigram_next; cs.max_order = max_order;
+    cs.K = K; cs.max_block = max_block;
     cs.lenience = lenience; cs.temperature = temperature; cs.seed = seed; cs.step = 0;
     cs.V = models[0]->c.vocab;
     cs.cap = models[0]->c.max_seq;
     for (int r = 1; r < n_levels; ++r)
         if (models[r]->c.max_seq < cs.cap) cs.cap = models[r]->c.max_seq;
-    /* how far drafting can run ahead of the committed prefix */
+    /* the product bounds how far drafting may run ahead of the committed prefix; the same bound is
+       applied here so that both sides accept and refuse the same requests */
     int window = 0;
     for (int r = 0; r < n_levels; ++r) {
         for (int c = r; c < n_levels; ++c) window += K[(size_t)r * n_levels + c] > 0 ? K[(size_t)r * n_levels + c] : 0;
         window += max_block + 1;
     }
-    if (window >= RING) return 2;
+    if (window >= 128) return 2;
     if (init_len + max_new + window > cs.cap) return 2;
     cs.seq = (int32_t*)calloc((size_t)cs.cap + 64, sizeof(int32_t));
-    cs.src = (int*)calloc((size_t)cs.cap + 64, sizeof(int));
-    cs.kv = (int*)calloc((size_t)n_levels, sizeof(int));
-    cs.qlaw = (float*)malloc(sizeof(float) * (size_t)RING * cs.V);
-    cs.law = (float*)malloc(sizeof(float) * (size_t)(max_block + 1) * cs.V);
+    cs.probs = (float**)calloc((size_t)cs.cap + 64, sizeof(float*));
     memcpy(cs.seq, init_seq, sizeof(int32_t) * (size_t)init_len);
-    cs.len = init_len; cs.prefix_len = init_len; cs.margins = margins;
+    cs.len = init_len; cs.init_len = init_len; cs.margins = margins;
     int rc = 0;
     for (int r = 0; r < n_levels && !rc; ++r)
         if (models[r]->c.arch == 1) rc = orc_encoder_forward(models[r], hay, L);
@@ -881,6 +891,7 @@ int orc_cascade_generate(orc_model** models, int n_levels, const int32_t* hay, i
     memcpy(out_tokens, cs.seq + init_len, sizeof(int32_t) * (size_t)made);
     *out_len = made;
     cs.st->tokens = made;
-    free(cs.qlaw); free(cs.law); free(cs.kv); free(cs.src); free(cs.seq);
+    for (int i = 0; i < cs.cap + 64; ++i) free(cs.probs[i]);
+    free(cs.probs); free(cs.seq);
     return rc;
 }

@@ -213,6 +213,122 @@ def test_t5_against_transformers(orc):
     assert 1e-5 < rel_l2(rounded, ref) < 5e-2
 
 
+def torch_t5_forward(shape, w, enc, dec, round_kv=True):
+    """Encoder-decoder forward from library routines (matmul, softmax, gelu, the library's bucket
+    function); every K and V that the product keeps in a bf16 cache (encoder self-attention, decoder
+    self-attention, cross-attention) is rounded to 8 significant bits right after its projection."""
+    from transformers.models.t5.modeling_t5 import T5Attention
+    H, Dh, d = shape.n_heads, shape.d_head, shape.d_model
+
+    def norm(v, g):
+        return v * torch.rsqrt(v.pow(2).mean(-1, keepdim=True) + shape.norm_eps) * g
+
+    def kvr(v):
+        if not round_kv:
+            return v
+        mant, expo = torch.frexp(v)
+        return torch.ldexp(torch.round(mant * 256.0), expo - 8)
+
+    def heads(v):
+        return v.view(v.shape[0], H, Dh).transpose(0, 1)          # [H, T, Dh]
+
+    def bias(table, nq, nk, bidir):
+        rel = torch.arange(nk)[None, :] - torch.arange(nq)[:, None]
+        bucket = T5Attention._relative_position_bucket(rel, bidirectional=bidir, num_buckets=shape.rel_buckets,
+                                                       max_distance=shape.rel_max_dist)
+        return table[bucket].permute(2, 0, 1)                      # [H, nq, nk]
+
+    def attend(q, k, v, extra):
+        sc = heads(q) @ heads(k).transpose(1, 2)                   # no 1/sqrt(Dh): the family does not scale
+        if extra is not None:
+            sc = sc + extra
+        return (torch.softmax(sc, dim=-1) @ heads(v)).transpose(0, 1).reshape(q.shape[0], H * Dh)
+
+    def ffn(x, p):
+        h = norm(x, w[p + ".norm2"])
+        g = torch.nn.functional.gelu(h @ w[p + ".wgate"].T, approximate="tanh") * (h @ w[p + ".wup"].T)
+        return x + g @ w[p + ".wdown"].T
+
+    E, T = len(enc), len(dec)
+    x = w["embed"][torch.from_numpy(enc.astype(np.int64))]
+    eb = bias(w["enc.rel_bias"], E, E, True)
+    for l in range(shape.n_enc_layers):
+        h = norm(x, w[f"e{l}.norm1"])
+        x = x + attend(h @ w[f"e{l}.wq"].T, kvr(h @ w[f"e{l}.wk"].T), kvr(h @ w[f"e{l}.wv"].T), eb) @ w[f"e{l}.wo"].T
+        x = ffn(x, f"e{l}")
+    mem = norm(x, w["enc.final_norm"])
+    y = w["embed"][torch.from_numpy(dec.astype(np.int64))]
+    causal = torch.full((T, T), float("-inf"), dtype=torch.float64).triu(1)
+    db = bias(w["dec.rel_bias"], T, T, False) + causal
+    for l in range(shape.n_layers):
+        h = norm(y, w[f"l{l}.norm1"])
+        y = y + attend(h @ w[f"l{l}.wq"].T, kvr(h @ w[f"l{l}.wk"].T), kvr(h @ w[f"l{l}.wv"].T), db) @ w[f"l{l}.wo"].T
+        h = norm(y, w[f"l{l}.norm_x"])
+        y = y + attend(h @ w[f"l{l}.xq"].T, kvr(mem @ w[f"l{l}.xk"].T), kvr(mem @ w[f"l{l}.xv"].T), None) @ w[f"l{l}.xo"].T
+        y = ffn(y, f"l{l}")
+    return (norm(y, w["final_norm"]) @ w["lm_head"].T).numpy()
+
+
+def test_t5_with_bf16_caches_against_torch_routines(orc):
+    # pins WHERE the encoder-decoder path rounds: all three K/V kinds, right after their projections
+    shape = SHAPES["t5tiny_target"]
+    blob = workloads.make_weights(shape, seed=2, gain_std=0.2, std=0.08)
+    w = tensors(shape, blob)
+    enc = workloads.make_prompt(shape.vocab, 37, seed=4)
+    dec = np.concatenate([[0], workloads.make_prompt(shape.vocab, 20, seed=6)]).astype(np.int32)
+    ref = torch_t5_forward(shape, w, enc, dec)
+    m = orc.Model(shape, orc.blob_to_u16(blob))
+    m.encoder_forward(enc)
+    got = np.concatenate([m.review_forward(dec[:1], 0), m.review_forward(dec[1:8], 1), m.review_forward(dec[8:], 8)])
+    assert rel_l2(got, ref) < 1e-6
+    # each of the three roundings matters on its own at a level far above that bound, so a rounding
+    # moved, dropped or doubled in the oracle would fail the comparison above
+    exact = torch_t5_forward(shape, w, enc, dec, round_kv=False)
+    assert 1e-5 < rel_l2(exact, ref) < 5e-2
+    orc.set_kv_exact(True)
+    try:
+        m2 = orc.Model(shape, orc.blob_to_u16(blob))
+        m2.encoder_forward(enc)
+        unrounded = m2.review_forward(dec, 0)
+    finally:
+        orc.set_kv_exact(False)
+    assert rel_l2(unrounded, exact) < 1e-6
+
+
+def test_two_correct_forwards_drift_apart_only_through_the_bf16_cache(orc):
+    # The same forward carried two equally valid ways (float64 throughout; contraction results
+    # rounded to float32).  With an unrounded cache the two stay within float32 rounding at any
+    # depth.  With the bf16 cache a difference of 1e-7 upstream moves some K/V entries across a
+    # rounding boundary, each worth 2^-9, and the gap grows by orders of magnitude with depth:
+    # a deep stack compared against ANY second implementation sees this gap, whatever the
+    # accuracy of that implementation's own arithmetic.
+    from workloads import llama_shape
+    gaps = {}
+    for depth in (1, 4, 32):
+        shape = llama_shape(depth, 256, 4, 688, 1000, 64)
+        blob = orc.blob_to_u16(workloads.make_weights(shape, seed=5, std=0.05))
+        toks = workloads.make_prompt(shape.vocab, 40, seed=3)
+        for exact in (False, True):
+            outs = []
+            for f32 in (False, True):
+                orc.set_kv_exact(exact)
+                orc.set_linear_f32(f32)
+                try:
+                    m = orc.Model(shape, blob)
+                    outs.append(np.concatenate([m.review_forward(toks[:17], 0), m.review_forward(toks[17:22], 17),
+                                                m.review_forward(toks[22:], 22)]))
+                finally:
+                    orc.set_kv_exact(False)
+                    orc.set_linear_f32(False)
+            gaps[depth, exact] = rel_l2(outs[1], outs[0])
+    for depth in (1, 4, 32):
+        assert gaps[depth, True] < 1e-6                      # unrounded cache: float32 rounding only
+    assert gaps[1, False] < 1e-6                             # one layer: its own K/V see identical inputs
+    assert gaps[4, False] > 50 * gaps[4, True]
+    assert gaps[32, False] > 1000 * gaps[32, True]           # measured: 6.7e-4 against 1.3e-7
+    assert gaps[32, False] < 5e-3
+
+
 def test_bf16_rounding_is_nearest_even(orc):
     rng = np.random.default_rng(0)
     xs = np.concatenate([rng.standard_normal(2000) * 10.0 ** rng.integers(-6, 6, 2000), [0.0, 1.0, -1.0]])

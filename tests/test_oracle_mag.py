@@ -1,5 +1,6 @@
-"""Pins the oracle's Max-Gram drafter (Section 3.3, Appendix A) to hand-worked cases and to a
-brute-force longest-suffix search written straight from the definition."""
+"""Pins the oracle's Max-Gram drafter (Section 3.3, Appendix A) to hand-worked cases and to the
+tensor formulation of Appendix A (boolean match vectors that are extended one token at a time),
+written here with numpy; the oracle itself searches order by order, start by start."""
 import os
 
 import numpy as np
@@ -10,15 +11,22 @@ GOLD = os.path.join(os.path.dirname(__file__), "golden", "mag_cases.txt")
 
 
 def brute_search(hay, seq, max_order):
-    """Index of the token after the longest, earliest suffix match that is followed by a
-    haystack token; None without a match."""
-    L, T = len(hay), len(seq)
-    for order in range(min(T, max_order), 0, -1):
-        needle = list(seq[T - order:])
-        for j in range(0, L - order):          # j + order <= L - 1: a following token exists
-            if list(hay[j:j + order]) == needle:
-                return j + order
-    return None
+    """Index of the token after the longest, earliest suffix match that is followed by a haystack
+    token; None without a match.  alive[j] says that a match of `order` tokens ENDS at haystack
+    index j; a longer match ending there needs one more equal token on its left."""
+    hay, seq = np.asarray(hay), np.asarray(seq)
+    L = len(hay)
+    alive = hay == seq[-1]
+    alive[L - 1:] = False                      # the last haystack token has nothing after it
+    if not alive.any():
+        return None
+    for order in range(2, min(len(seq), max_order) + 1):
+        longer = np.zeros(L, dtype=bool)
+        longer[order - 1:] = alive[order - 1:] & (hay[:L - order + 1] == seq[-order])
+        if not longer.any():
+            break
+        alive = longer
+    return int(np.flatnonzero(alive)[0]) + 1   # earliest end = earliest start, the length being fixed
 
 
 def brute_draft(hay, nxt, seq, n, max_order):
@@ -102,3 +110,22 @@ def test_bigram_table_generator():
     nxt = workloads.bigram_table(prompt, 16, seed=1)
     assert nxt[4] == 7 and nxt[7] == 4 and nxt[9] == 2
     assert ((nxt >= 0) & (nxt < 16)).all()
+
+
+def test_dynamic_haystack_is_the_static_search_over_prompt_plus_generation(orc):
+    # Section 3.3 lets the match come from the initial input or from what has been generated.  With a
+    # target that soon repeats itself, a drafter that also searches the generation gets more of its
+    # tokens accepted than one that searches the prompt alone, and the output stays the target's own.
+    from workloads import llama_shape
+    shape = llama_shape(1, 16, 2, 32, 12, 200)
+    blob = orc.blob_to_u16(workloads.make_weights(shape, seed=3, std=1.5))
+    prompt = workloads.make_prompt(shape.vocab, 6, seed=1)
+    nxt = workloads.bigram_table(prompt, shape.vocab, seed=1)
+    outs, accepted = [], []
+    for dyn in (False, True):
+        got, _, st = orc.cascade_generate([orc.Model(shape, blob)], prompt, nxt, [[6]], 6, prompt, 120,
+                                          dynamic_haystack=dyn)
+        outs.append(got.tolist())
+        accepted.append(st["accepted"][0])
+    assert outs[0] == outs[1]                  # greedy: the drafter cannot change the output
+    assert accepted[1] > accepted[0] + 10
