@@ -141,8 +141,10 @@ csd_status csd_model_profile_read(csd_model* m, void* stream, csd_profile* out);
 size_t csd_linear_workspace_bytes(int m, int N, int K);
 /* Which kernel the contraction uses, process-wide: 0 = automatic choice per shape, 1 = the
  * CUDA-core kernel (128-bit streaming loads, fp32 FMA), 2 = the tensor-core kernel (TMA-staged
- * weights, tcgen05.mma with fp32 accumulators in tensor memory) wherever it applies (K >= 64).
- * Both give the same result up to fp32 summation order; the switch exists to measure them. */
+ * weights, tcgen05.mma with fp32 accumulators in tensor memory) with equal shares of (tile, K block)
+ * units per CTA wherever it applies (K >= 64), 3 = the tensor-core kernel in which every CTA owns
+ * whole output columns over all of K (no partial sums between CTAs) wherever it applies, 2 elsewhere.
+ * All give the same result up to fp32 summation order; the switch exists to measure them. */
 csd_status csd_set_gemm_path(int path);
 /* Which kernel the block attention uses, process-wide: 0 = automatic (tensor cores, mma.sync on
  * TMA-staged K/V tiles, for head dimensions 64 and 128; the CUDA-core kernel for 32), 1 = always

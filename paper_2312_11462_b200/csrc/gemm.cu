@@ -335,12 +335,36 @@ bool linear_uses_tensor_cores(int m, int N, int K, bool dual) {
     return path != 1 && tc_supported(m, N, K, dual) && (path == 2 || (long long)N * K >= AUTO_TC_MIN_WEIGHTS);
 }
 
+// Which tensor-core kernel.  One tcgen05.mma reads 128 rows of shared memory for its wide operand
+// and takes about 80 cycles whatever part of them is a CTA's own range, so the row-range kernel
+// keeps up with the memory stream only where a range fills most of those rows.  Measured on the 7B
+// shapes at 5 rows, each GEMM alone: 84 rows of the fused q|k|v projection 19 us against 20 with
+// equal shares and a fix-up pass, 109 rows of the vocabulary projection equal, the 28 rows of the
+// projections back to d_model 35 us against 17; inside a forward, where consecutive kernels overlap,
+// the row-range kernel on q|k|v costs 5 us per layer more than it saves.  It is therefore chosen
+// only on request (path 3) and stays as the comparison kernel without any cross-CTA traffic.
+bool linear_uses_row_ranges(int m, int N, int K, bool dual) {
+    if (!linear_uses_tensor_cores(m, N, K, dual) || !rs_supported(m, N, K, dual)) return false;
+    return gemm_path() == 3;
+}
+
+int linear_ssq_pieces(int m, int N, int K, bool dual) {
+    return linear_uses_row_ranges(m, N, K, dual) ? rs_ssq_pieces(m, N, K, dual) : 4 * ((N + 127) / 128);
+}
+
+int linear_ssq_capacity(int N) {
+    const int sms = tc_sm_count(), per = (N + sms - 1) / sms, T = (per + 127) / 128;
+    const int a = 4 * ((N + 127) / 128), b = sms * T * 4;
+    return a > b ? a : b;
+}
+
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
     if (!a.W || !a.X || !a.Y || a.m < 1 || a.m > CSD_MAX_ROWS || a.N < 1 || a.K < 8 || (a.K & 7))
         return CSD_ERR_INVALID_ARG;
     const bool dual = a.W2 != nullptr;
     if (dual != (a.epilogue == EPI_SWIGLU || a.epilogue == EPI_GEGLU)) return CSD_ERR_INVALID_ARG;
     if ((((uintptr_t)a.W) & 15) || (dual && (((uintptr_t)a.W2) & 15))) return CSD_ERR_INVALID_ARG;
+    if (a.xs && linear_uses_row_ranges(a.m, a.N, a.K, dual)) return launch_linear_rs(a, st);
     if (a.xs && linear_uses_tensor_cores(a.m, a.N, a.K, dual)) return launch_linear_tc(a, st);
     if ((((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
     const LinearPlan pl = plan_linear(a.m, a.N, a.K, dual);
@@ -367,7 +391,7 @@ csd_status launch_linear(const LinearArgs& a, cudaStream_t st) {
 using namespace csd;
 
 extern "C" csd_status csd_set_gemm_path(int path) {
-    if (path < 0 || path > 2) return CSD_ERR_INVALID_ARG;
+    if (path < 0 || path > 3) return CSD_ERR_INVALID_ARG;
     set_gemm_path(path);
     return CSD_OK;
 }

@@ -28,7 +28,7 @@ struct LinearArgs {
     __nv_bfloat16* out_xs = nullptr;     // three-term split of (Y * out_gain), [3m][out_ld]
     int out_ld = 0;
     const __nv_bfloat16* out_gain = nullptr;
-    float* out_ssq = nullptr;            // [4 * ceil(N/128)][m] pieces of the sums of squares of the rows of Y
+    float* out_ssq = nullptr;            // [linear_ssq_pieces(...)][m] pieces of the sums of squares of the rows of Y
 };
 
 int split_rows(int m);                   // 16, 32, 48 or 64 operand rows hold the 3m terms
@@ -38,5 +38,8 @@ size_t linear_scratch_bytes(int m, int N, int K, bool dual);
 int linear_ticket_count(int N);
 csd_status launch_linear(const LinearArgs& a, cudaStream_t st);
 bool linear_uses_tensor_cores(int m, int N, int K, bool dual);   // the kernel launch_linear would pick (given a.xs)
+bool linear_uses_row_ranges(int m, int N, int K, bool dual);     // ... and which of the two tensor-core kernels
+int linear_ssq_pieces(int m, int N, int K, bool dual);           // out_ssq pieces that launch writes
+int linear_ssq_capacity(int N);                                  // upper bound of the above over m, K
 
 }  // namespace csd

@@ -267,28 +267,31 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         //      the first ring-full of weight tiles goes out before the dependency wait; the rows'
         //      terms follow after it.
         if (lane == 0) {
+            // (all index arithmetic of this thread is incremental: a division per stage costs more
+            // than the copy instructions it feeds)
             const int pre = items < p.stages ? items : p.stages;
+            int tile = (int)(u0 / p.nkb), kb = (int)(u0 % p.nkb);
+            const int kb0 = kb;
             for (int i = 0; i < pre; ++i) {
-                const unsigned u = u0 + i;
-                const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
                 unsigned char* dst = ring + (size_t)i * STAGE;
                 mbar_expect_tx(&ctl->full[i], (uint32_t)STAGE);
                 tma_load_2d(dst, &tmW, &ctl->full[i], kb * KS * KB, tile * TILE_N);
                 if (DUAL) tma_load_2d(dst + STAGE_BYTES, &tmW2, &ctl->full[i], kb * KB, tile * TILE_N);
                 if (KS == 2) tma_load_2d(dst + STAGE_BYTES, &tmW, &ctl->full[i], (kb * KS + 1) * KB, tile * TILE_N);   // past K: zero fill
+                if (++kb == p.nkb) { kb = 0; ++tile; }
             }
             asm volatile("griddepcontrol.wait;" ::: "memory");
+            int kx = kb0;
             for (int i = 0; i < pre; ++i) {
-                const int kb = (int)((u0 + i) % p.nkb);
 #pragma unroll
                 for (int j = 0; j < KS; ++j)
-                    tma_load_2d(ring + (size_t)i * STAGE + WB + j * XBYTES, &tmX, &ctl->full[i], (kb * KS + j) * KB, 0);
+                    tma_load_2d(ring + (size_t)i * STAGE + WB + j * XBYTES, &tmX, &ctl->full[i], (kx * KS + j) * KB, 0);
+                if (++kx == p.nkb) kx = 0;
             }
+            int s = 0;
+            uint32_t ph = 0;                      // parity of the phase of empty[s] that frees slot s next
             for (int i = pre; i < items && !*abort_flag; ++i) {
-                const int s = i % p.stages;
-                if (!mbar_wait(&ctl->empty[s], ((i / p.stages) - 1) & 1)) { *abort_flag = 1; break; }
-                const unsigned u = u0 + i;
-                const int tile = (int)(u / p.nkb), kb = (int)(u % p.nkb);
+                if (!mbar_wait(&ctl->empty[s], ph)) { *abort_flag = 1; break; }
                 unsigned char* dst = ring + (size_t)s * STAGE;
                 mbar_expect_tx(&ctl->full[s], (uint32_t)STAGE);
                 tma_load_2d(dst, &tmW, &ctl->full[s], kb * KS * KB, tile * TILE_N);
@@ -297,34 +300,39 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 #pragma unroll
                 for (int j = 0; j < KS; ++j)
                     tma_load_2d(dst + WB + j * XBYTES, &tmX, &ctl->full[s], (kb * KS + j) * KB, 0);
+                if (++kb == p.nkb) { kb = 0; ++tile; }
+                if (++s == p.stages) { s = 0; ph ^= 1u; }
             }
         }
     } else if (warp == 1) {
         // ---- MMA issuer: one accumulator set per segment (the part of a tile inside this CTA's range)
         if (lane == 0) {
-            int i = 0;
+            int i = 0, s = 0;
+            uint32_t ph = 0;                      // parity of the phase of full[s] that fills slot s next
+            int kb_begin = (int)(u0 % p.nkb);
+            const uint64_t desc0 = smem_desc_sw128(smem_u32(ring));   // descriptors differ in the address field only
             for (int seg = 0; i < items && !*abort_flag; ++seg) {
                 const int b = seg & 1;
-                const int kb_begin = (int)((u0 + i) % p.nkb);
                 const int seg_len = min(p.nkb - kb_begin, items - i);
+                kb_begin = 0;                     // later segments start at a tile's first K block
                 if (!mbar_wait(&ctl->acc_empty[b], ((seg >> 1) & 1) ^ 1)) { *abort_flag = 1; break; }
                 tc_fence_after();
                 const uint32_t d0 = tmem + (uint32_t)(b * ACC_COLS);
                 for (int j = 0; j < seg_len; ++j, ++i) {
-                    const int s = i % p.stages;
-                    if (!mbar_wait(&ctl->full[s], (i / p.stages) & 1)) { *abort_flag = 1; break; }
+                    if (!mbar_wait(&ctl->full[s], ph)) { *abort_flag = 1; break; }
                     tc_fence_after();
-                    const uint32_t a_addr = smem_u32(ring + (size_t)s * STAGE);
-                    const uint32_t b_addr = a_addr + WB;
+                    const uint64_t ad = desc0 + (uint64_t)(((uint32_t)s * (uint32_t)STAGE) >> 4);
+                    const uint64_t bd = ad + (WB >> 4);
 #pragma unroll
                     for (int h = 0; h < KS; ++h)
 #pragma unroll
                         for (int k = 0; k < KB / 16; ++k) {
-                            const uint64_t bd = smem_desc_sw128(b_addr + h * XBYTES + k * 32);
-                            tc_mma(d0, smem_desc_sw128(a_addr + h * STAGE_BYTES + k * 32), bd, IDESC, (j | h | k) != 0);
-                            if (DUAL) tc_mma(d0 + NPAD, smem_desc_sw128(a_addr + STAGE_BYTES + k * 32), bd, IDESC, (j | k) != 0);
+                            const uint64_t bdk = bd + ((h * XBYTES) >> 4) + 2 * k;
+                            tc_mma(d0, ad + ((h * STAGE_BYTES) >> 4) + 2 * k, bdk, IDESC, (j | h | k) != 0);
+                            if (DUAL) tc_mma(d0 + NPAD, ad + (STAGE_BYTES >> 4) + 2 * k, bdk, IDESC, (j | k) != 0);
                         }
                     tc_commit(&ctl->empty[s]);          // stage reusable once these MMAs have read it
+                    if (++s == p.stages) { s = 0; ph ^= 1u; }
                 }
                 if (*abort_flag) break;
                 tc_commit(&ctl->acc_full[b]);           // this segment's accumulators are complete
@@ -569,6 +577,19 @@ static void pdl_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, dim3 
     cfg.attrs = attr; cfg.numAttrs = 1;
 }
 
+// Splits a.X (times a.gain) into a.xs and writes the sum-of-squares pieces into a.ssq.
+csd_status launch_split_rows(const LinearArgs& a, cudaStream_t st) {
+    if (!a.X || (((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
+    if (a.gain && !a.ssq) return CSD_ERR_INVALID_ARG;
+    cudaLaunchConfig_t cfg;
+    cudaLaunchAttribute attr[1];
+    pdl_config(cfg, attr, dim3((unsigned)split_ssq_entries(a.K), (unsigned)a.m), dim3(128), 0, st);
+    CSD_CUDA(cudaLaunchKernelEx(&cfg, split_rows_kernel, a.X, a.ldx, a.K, a.m, a.gain, a.xs,
+                                a.gain ? a.ssq : (float*)nullptr));
+    count_launch();
+    return CSD_OK;
+}
+
 template <int M, bool DUAL>
 static csd_status launch_tc(const CUtensorMap& tw, const CUtensorMap& tw2, const CUtensorMap& tx, const TcParams& tp,
                             const TcPlan& pl, cudaStream_t st) {
@@ -606,14 +627,8 @@ csd_status launch_linear_tc(const LinearArgs& a, cudaStream_t st) {
     if (!tensor_map_2d(a.xs, 3 * a.m, a.K, pl.npad, &tx)) return CSD_ERR_UNSUPPORTED;
     int ssq_cnt = a.ssq_cnt;
     if (!a.xs_ready) {
-        if (!a.X || (((uintptr_t)a.X) & 15) || (a.ldx & 3)) return CSD_ERR_INVALID_ARG;
-        if (a.gain && !a.ssq) return CSD_ERR_INVALID_ARG;
-        cudaLaunchConfig_t cfg;
-        cudaLaunchAttribute attr[1];
-        pdl_config(cfg, attr, dim3((unsigned)split_ssq_entries(a.K), (unsigned)a.m), dim3(128), 0, st);
-        CSD_CUDA(cudaLaunchKernelEx(&cfg, split_rows_kernel, a.X, a.ldx, a.K, a.m, a.gain, a.xs,
-                                    a.gain ? a.ssq : (float*)nullptr));
-        count_launch();
+        const csd_status s = launch_split_rows(a, st);
+        if (s != CSD_OK) return s;
         ssq_cnt = split_ssq_entries(a.K);
     }
     TcParams tp;

@@ -168,7 +168,7 @@ static WsLayout ws_layout(const csd_model_config& c) {
     L.xs_x = put(3 * R * d * 2);
     L.xs_attn = put(3 * R * di * 2);
     L.xs_act = put(3 * R * ff * 2);
-    L.ssq_x = put(4 * ((d + 127) / 128) * R * 4);
+    L.ssq_x = put((size_t)linear_ssq_capacity((int)d) * R * 4);
     if (c.arch == 0) {
         L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
         L.rope_s = put((size_t)c.max_seq * (Dh / 2) * 4);
@@ -228,6 +228,7 @@ static csd_status linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat
             a.ssq = const_cast<float*>(o->ssq_in); a.ssq_cnt = o->ssq_cnt;
         }
         a.out_xs = o->out_xs; a.out_ld = o->out_ld; a.out_gain = o->out_gain; a.out_ssq = o->out_ssq;
+        if (o->out_ssq == M->ssq_x) M->ssq_x_cnt = linear_ssq_pieces(m, N, K, W2 != nullptr);
     }
     ProfScope ps(M, 0, st);
     if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
@@ -265,10 +266,9 @@ static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, c
                                bool x_in = false, const __nv_bfloat16* next_gain = nullptr, int next_N = 0,
                                bool next_dual = false, bool* x_out = nullptr) {
     const int d = M->cfg.d_model, ff = M->cfg.d_ff;
-    const int cnt_d = 4 * ((d + 127) / 128);
     const bool tc_up = linear_uses_tensor_cores(m, ff, d, true), tc_down = linear_uses_tensor_cores(m, d, ff, false);
     LinOpt up;
-    if (x_in) { up.xs_in = M->xs_x; up.ssq_in = M->ssq_x; up.ssq_cnt = cnt_d; }
+    if (x_in) { up.xs_in = M->xs_x; up.ssq_in = M->ssq_x; up.ssq_cnt = M->ssq_x_cnt; }
     const bool act_ready = tc_up && tc_down;
     if (act_ready) { up.out_xs = M->xs_act; up.out_ld = ff; }
     CSD_TRY(linear(M, y.wgate, y.wup, ff, d, X, d, m, y.norm2, M->act, ff, M->cfg.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, st, &up));
@@ -477,7 +477,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
     // x_ready: M->xs_x / M->ssq_x hold the residual rows (times the gain of the norm that reads them
     // next) in three-term form, written by the epilogue of the GEMM that produced the rows
     bool x_ready = false;
-    const int ff = c.d_ff, cnt_d = 4 * ((d + 127) / 128);
+    const int ff = c.d_ff;
     const bool tc_o = linear_uses_tensor_cores(m, d, di, false);
     for (int l = 0; l < c.n_layers; ++l) {
         const LayerW& y = M->dec[l];
@@ -485,7 +485,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
         {
             LinOpt qo;
-            if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = cnt_d; }
+            if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = M->ssq_x_cnt; }
             CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         }
         AttnArgs a;
@@ -508,7 +508,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         CSD_TRY(linear(M, y.wo, nullptr, d, di, M->attn, di, m, nullptr, M->x, d, EPI_ADD, st, &oo));
         if (c.arch == 1) {
             LinOpt xq;
-            if (x_ready) { xq.xs_in = M->xs_x; xq.ssq_in = M->ssq_x; xq.ssq_cnt = cnt_d; }
+            if (x_ready) { xq.xs_in = M->xs_x; xq.ssq_in = M->ssq_x; xq.ssq_cnt = M->ssq_x_cnt; }
             CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st, &xq));
             AttnArgs x;
             x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
@@ -532,7 +532,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         CSD_TRY(feed_forward(M, y, M->x, m, st, x_ready, next_gain, next_N, false, &x_ready));
     }
     LinOpt ho;
-    if (x_ready) { ho.xs_in = M->xs_x; ho.ssq_in = M->ssq_x; ho.ssq_cnt = cnt_d; }
+    if (x_ready) { ho.xs_in = M->xs_x; ho.ssq_in = M->ssq_x; ho.ssq_cnt = M->ssq_x_cnt; }
     CSD_TRY(linear(M, M->lm_head, nullptr, V, d, M->x, d, m, M->final_norm, logits_out_dev, V, EPI_STORE, st, &ho));
     CSD_CUDA(cudaGetLastError());
     return CSD_OK;

@@ -32,7 +32,8 @@ struct csd_model {
     float* ssq_tmp = nullptr;           // pieces of the rows' sums of squares written with it
     // activations handed from kernel to kernel in three-term form (tensor-core path)
     __nv_bfloat16 *xs_x = nullptr, *xs_attn = nullptr, *xs_act = nullptr;   // [3*17][d], [3*17][d_inner], [3*17][d_ff]
-    float* ssq_x = nullptr;             // [4 * ceil(d/128)][17] pieces of the sums of squares of the residual rows
+    float* ssq_x = nullptr;             // [ssq_x_cnt][rows] pieces of the sums of squares of the residual rows
+    int ssq_x_cnt = 0;                  // pieces the GEMM that last produced the residual rows wrote
     int* status = nullptr;
     // optional per-kernel-class timing (csd_model_profile): event pairs around every launch
     bool prof = false;

@@ -51,7 +51,7 @@ def test_7b_shaped_cascade_and_logits(b, orc):
         assert np.abs(g - r).max() <= LOGIT_MAX_ABS
 
 
-@pytest.mark.parametrize("path", [1, 2], ids=["cuda-core", "tensor-core"])
+@pytest.mark.parametrize("path", [1, 2, 3], ids=["cuda-core", "tensor-core", "tensor-core-row-ranges"])
 def test_7b_width_shallow_stack(b, orc, path):
     # the 7B layer shapes (d 4096, 32 heads x 128, ffn 11008, vocabulary 32000) in a 3-layer stack
     shape = llama_shape(3, 4096, 32, 11008, 32000, 64)

@@ -8,9 +8,10 @@ from gpu_util import rel_l2, require_gpu
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=[1, 2], ids=["cuda-core", "tensor-core"])
+@pytest.fixture(scope="module", params=[1, 2, 3], ids=["cuda-core", "tensor-core", "tensor-core-row-ranges"])
 def b(request):
-    """Every test here runs once per GEMM kernel: 128-bit loads + fp32 FMA, and TMA + tcgen05."""
+    """Every test here runs once per GEMM kernel: 128-bit loads + fp32 FMA, TMA + tcgen05 with equal
+    shares of (tile, K block) units, and TMA + tcgen05 with whole output columns per CTA."""
     require_gpu()
     from paper_2312_11462_b200 import binding
     binding.csd_set_gemm_path(request.param)
@@ -46,3 +47,10 @@ def test_layer_shapes(b, orc, m):
 def test_7b_layer_shapes(b, orc, N, K):
     for m in (5, 17):
         case(b, orc, m, N, K, seed=m)
+
+
+def test_head_shape_and_uneven_ranges(b, orc):
+    # the vocabulary projection (two row ranges per CTA in the row-range kernel) and row counts
+    # that leave ranges of unequal length, a K tail and fewer K blocks than a stage holds
+    for m, N, K in ((5, 32000, 4096), (3, 20011, 1032), (8, 2371, 4104), (2, 2368, 72)):
+        case(b, orc, m, N, K, seed=N + m)
