@@ -116,9 +116,10 @@ def set_kv_exact(on: bool) -> None:
     lib().orc_set_kv_exact(int(on))
 
 
-def set_linear_f32(on: bool) -> None:
-    """Test hook: round every contraction result to fp32 (a second correct way to do the sums)."""
-    lib().orc_set_linear_f32(int(on))
+def set_linear_f32(mode) -> None:
+    """Test hook: 1/True rounds every contraction result to fp32, 2 runs the contractions in fp32
+    throughout (two more correct ways to do the sums), 0/False restores the fp64 sums."""
+    lib().orc_set_linear_f32(int(mode))
 
 
 def top2_margin(logits) -> float:

@@ -409,8 +409,9 @@ void orc_model_destroy(orc_model* m) {
     free(m);
 }
 
-/* Test hook: with `on`, every result of a contraction is rounded to fp32 before it is used.  That
-   is a second, equally correct way to carry the arithmetic; the tests use it to measure how far two
+/* Test hook: with 1, every result of a contraction is rounded to fp32 before it is used; with 2,
+   the contraction itself runs in fp32 (fp32 operands, products and running sum, in index order).
+   Both are equally correct ways to carry the arithmetic; the tests use them to measure how far two
    correct implementations drift apart once both round K/V to bf16. */
 static int g_linear_f32 = 0;
 void orc_set_linear_f32(int on) { g_linear_f32 = on; }
@@ -422,6 +423,12 @@ static void linear(const uint16_t* W, int N, int K, const double* X, int m, doub
         const uint16_t* w = W + (size_t)n * K;
         for (int r = 0; r < m; ++r) {
             const double* x = X + (size_t)r * K;
+            if (g_linear_f32 == 2) {
+                float acc32 = 0.f;
+                for (int k = 0; k < K; ++k) acc32 += (float)bf16_to_double(w[k]) * (float)x[k];
+                Y[(size_t)r * N + n] = (double)acc32;
+                continue;
+            }
             double acc = 0.0;
             for (int k = 0; k < K; ++k) acc += bf16_to_double(w[k]) * x[k];
             Y[(size_t)r * N + n] = g_linear_f32 ? (double)(float)acc : acc;

@@ -183,6 +183,8 @@ accept_decide_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
         if (threadIdx.x != 0) return;
         int n = 0;
         while (n < k && tok[n] == s_arg[n]) ++n;
+        for (int i = 0; i < k; ++i)             // a drafted id outside the vocabulary is rejected and recorded
+            if (tok[i] < 0 || tok[i] >= V) set_status(status, CSD_ERR_BAD_TOKEN);
         n_acc[row] = n;
         out_tok[row] = s_arg[n];
         ri.n = n;

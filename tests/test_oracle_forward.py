@@ -329,6 +329,38 @@ def test_two_correct_forwards_drift_apart_only_through_the_bf16_cache(orc):
     assert gaps[32, False] < 5e-3
 
 
+def test_an_all_fp32_forward_drifts_further_and_levels_off(orc):
+    # The same comparison with the second forward carried in fp32 throughout (fp32 operands,
+    # products and running sums): the kind of implementation a GPU path with fp32 accumulation is.
+    # Its own arithmetic differs from the fp64 sums by a few 1e-7 per contraction, yet behind the
+    # bf16 cache the logits end up 1e-3 apart in a deep stack, and the gap levels off with depth
+    # instead of compounding.
+    from workloads import llama_shape
+    gap, exact_gap = {}, {}
+    for depth in (2, 8, 32):
+        shape = llama_shape(depth, 256, 4, 688, 1000, 64)
+        blob = orc.blob_to_u16(workloads.make_weights(shape, seed=5, std=0.05))
+        toks = workloads.make_prompt(shape.vocab, 40, seed=3)
+        for exact in (False, True):
+            outs = []
+            for mode in (0, 2):
+                orc.set_kv_exact(exact)
+                orc.set_linear_f32(mode)
+                try:
+                    m = orc.Model(shape, blob)
+                    outs.append(np.concatenate([m.review_forward(toks[:17], 0), m.review_forward(toks[17:22], 17),
+                                                m.review_forward(toks[22:], 22)]))
+                finally:
+                    orc.set_kv_exact(False)
+                    orc.set_linear_f32(0)
+            (exact_gap if exact else gap)[depth] = rel_l2(outs[1], outs[0])
+    for depth in (2, 8, 32):
+        assert exact_gap[depth] < 2e-6                       # fp32 sums alone: rounding level
+        assert gap[depth] > 20 * exact_gap[depth]            # the bf16 cache multiplies the difference
+    assert gap[32] < 5e-3
+    assert gap[32] < 4 * gap[8]                              # levels off: no compounding with depth
+
+
 def test_bf16_rounding_is_nearest_even(orc):
     rng = np.random.default_rng(0)
     xs = np.concatenate([rng.standard_normal(2000) * 10.0 ** rng.integers(-6, 6, 2000), [0.0, 1.0, -1.0]])

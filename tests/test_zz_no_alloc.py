@@ -47,6 +47,28 @@ def test_matches_the_workspace_entry_point_twice(b, rows, k, V, temperature):
     assert torch.equal(a1[0], a2[0]) and torch.equal(a1[1], a2[1])
 
 
+def test_allocates_nothing_and_takes_empty_and_greedy_calls(b):
+    t, d, tok = workloads.accept_case(32, 4, 32000, 0.5, seed=9, device="cuda")
+    out = outputs(32)
+    b.csd_spec_accept_static(t, d, tok, 1.0, out=out)           # the first call on a device looks the scratch up
+    torch.cuda.synchronize()
+    free_before = torch.cuda.mem_get_info()[0]
+    for step in range(3):
+        b.csd_spec_accept_static(t, d, tok, 1.0, step=step, out=out)
+    torch.cuda.synchronize()
+    assert torch.cuda.mem_get_info()[0] == free_before          # no device memory was taken
+    # greedy review with draft logits present (they are ignored), against the workspace entry point
+    want = b.csd_spec_accept(t, d, tok, 0.0)
+    got = b.csd_spec_accept_static(t, d, tok, 0.0, out=outputs(32))
+    assert torch.equal(got[0], want[0]) and torch.equal(got[1], want[1])
+    # no rows: nothing to do, nothing touched
+    keep = outputs(4)
+    code = b.lib.csd_spec_accept_static(t.data_ptr(), None, None, tok.data_ptr(), 0, 4, 32000, 1.0, 1.0, 0, 0,
+                                        keep[0].data_ptr(), keep[1].data_ptr(), None)
+    torch.cuda.synchronize()
+    assert code == 0 and (keep[0] == -7).all() and (keep[1] == -7).all()
+
+
 def test_refuses_what_does_not_fit_and_bad_arguments(b):
     cap = b.lib.csd_spec_accept_static_capacity()
     assert cap == 2 << 20
