@@ -109,12 +109,14 @@ csd_status csd_model_destroy(csd_model* m);
  * cross-attention K/V of every decoder layer.  Must precede csd_review_forward. */
 csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int n, void* stream);
 
-/* The review forward: "reviewed by a target model in parallel ... in one single run" (Sections
- * 1-2).  One pass over m rows (1 <= m <= max_rows) at positions kv_len .. kv_len+m-1: reads cache
- * rows [0, kv_len), OVERWRITES rows [kv_len, kv_len+m), writes logits_out_dev [m, vocab] fp32
- * row-major; row r is the model's next-token law after position kv_len+r, causal inside the
- * block.  The caller commits accepted positions by passing a larger kv_len next time; rejected
- * rows are simply overwritten (rollback is free). */
+/* The review forward: the larger model scores all drafted positions of a block in one pass
+ * (Sections 1-2).  One pass over m rows (1 <= m <= max_rows) at positions kv_len .. kv_len+m-1:
+ * reads cache rows [0, kv_len), OVERWRITES rows [kv_len, kv_len+m), writes logits_out_dev
+ * [m, vocab] fp32 row-major; row r is the model's next-token law after position kv_len+r, causal
+ * inside the block.  The caller commits accepted positions by passing a larger kv_len next time;
+ * rejected rows are simply overwritten (rollback is free).  logits_out_dev == NULL: the block is
+ * only appended to the cache (prompt prefill, catching up) and the vocabulary projection is
+ * skipped. */
 csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
                               float* logits_out_dev, void* stream);
 

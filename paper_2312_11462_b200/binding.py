@@ -157,9 +157,13 @@ class Model:
         _check("csd_encoder_forward", lib.csd_encoder_forward(self.h, _ptr(enc_tokens), enc_tokens.numel(), _stream()))
 
     def csd_review_forward(self, block_tokens: torch.Tensor, kv_len: int,
-                           logits_out: Optional[torch.Tensor] = None) -> torch.Tensor:
+                           logits_out: Optional[torch.Tensor] = None, append_only: bool = False):
+        """Returns the logits [m, vocab]; with append_only the block only enters the cache (no logits)."""
         assert block_tokens.dtype == torch.int32 and block_tokens.is_cuda
         m = block_tokens.numel()
+        if append_only:
+            _check("csd_review_forward", lib.csd_review_forward(self.h, _ptr(block_tokens), m, kv_len, None, _stream()))
+            return None
         if logits_out is None:
             logits_out = torch.empty(m, self.shape.vocab, dtype=torch.float32, device=block_tokens.device)
         _check("csd_review_forward",

@@ -3,6 +3,7 @@
 // the base case.  Tokens, logits and laws stay on the device; per review the host reads back
 // two integers (accepted count, output token).
 #include <chrono>
+#include <mutex>
 #include <string.h>
 #include <vector>
 #include "model.cuh"
@@ -32,6 +33,65 @@ static CascadeWs cascade_layout(int V, int max_block, int cap, int L, int max_or
     return w;
 }
 
+// Host-side resources of a generation (a small block of mapped pinned memory for the results of
+// the accept kernels, three events): created once per device and kept, so that a call creates and
+// frees nothing; a second call that overlaps the first on the same device makes its own.
+struct HostKit {
+    int32_t* pinned = nullptr; int32_t* mapped = nullptr; cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+    bool pooled = false;
+};
+constexpr int KIT_WORDS = 2 + CSD_MAX_ROWS + 64, KIT_DEVICES = 64;
+static std::mutex g_kit_mu;
+static HostKit g_kit[KIT_DEVICES];
+static bool g_kit_busy[KIT_DEVICES];
+
+static void kit_free(HostKit& k) {
+    for (cudaEvent_t& e : k.ev) { if (e) cudaEventDestroy(e); e = nullptr; }
+    if (k.pinned) cudaFreeHost(k.pinned);
+    k.pinned = nullptr; k.mapped = nullptr;
+}
+static csd_status kit_make(HostKit& k) {
+    if (cudaHostAlloc((void**)&k.pinned, (size_t)KIT_WORDS * 4, cudaHostAllocMapped) != cudaSuccess ||
+        cudaHostGetDevicePointer((void**)&k.mapped, k.pinned, 0) != cudaSuccess || !k.mapped) {
+        const csd_status s = note_cuda(cudaGetLastError());
+        kit_free(k);
+        return s != CSD_OK ? s : CSD_ERR_CUDA;
+    }
+    for (cudaEvent_t& e : k.ev)
+        if (cudaEventCreate(&e) != cudaSuccess) { const csd_status s = note_cuda(cudaGetLastError()); kit_free(k); return s; }
+    return CSD_OK;
+}
+static csd_status kit_acquire(HostKit& out) {
+    int dev = 0;
+    CSD_CUDA(cudaGetDevice(&dev));
+    std::lock_guard<std::mutex> lk(g_kit_mu);
+    if (dev >= 0 && dev < KIT_DEVICES && !g_kit_busy[dev]) {
+        if (!g_kit[dev].pinned) {
+            const csd_status s = kit_make(g_kit[dev]);
+            if (s != CSD_OK) return s;
+        }
+        g_kit_busy[dev] = true;
+        out = g_kit[dev];
+        out.pooled = true;
+        return CSD_OK;
+    }
+    out = HostKit{};
+    return kit_make(out);
+}
+static void kit_release(HostKit& k) {
+    if (!k.pinned) return;
+    if (k.pooled) {
+        int dev = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess) dev = -1;
+        std::lock_guard<std::mutex> lk(g_kit_mu);
+        for (int d = 0; d < KIT_DEVICES; ++d)
+            if (g_kit[d].pinned == k.pinned) g_kit_busy[d] = false;
+    } else {
+        kit_free(k);
+    }
+    k.pinned = nullptr;
+}
+
 struct Gen {
     csd_model* const* models; int n_levels; const int32_t* K; int max_block; float lenience, temperature;
     uint64_t seed, step = 0; csd_mag* mag = nullptr; int V, cap;
@@ -43,9 +103,10 @@ struct Gen {
     cudaEvent_t ev_decode; bool decode_marked = false;
 };
 
-// forward `cnt` rows of level r starting at sequence position `from`; logits land in g.law
-static csd_status forward(Gen& g, int r, int from, int cnt) {
-    csd_status s = csd_review_forward(g.models[r], g.seq + from, cnt, from, g.law, g.stream);
+// forward `cnt` rows of level r starting at sequence position `from`; logits land in g.law, or
+// nowhere when nobody reads them (prompt prefill, catch-up chunks before the reviewed block)
+static csd_status forward(Gen& g, int r, int from, int cnt, bool want_logits = true) {
+    csd_status s = csd_review_forward(g.models[r], g.seq + from, cnt, from, want_logits ? g.law : nullptr, g.stream);
     g.st->forwards[r] += 1;
     return s;
 }
@@ -61,7 +122,7 @@ static csd_status review(Gen& g, int r, int P, int nd) {
         cnt = P + nd - from;
         if (cnt > maxrows) cnt = (from + maxrows <= P - 1) ? maxrows : (P - 1) - from;
         CSD_CUDA(cudaGetLastError());
-        csd_status s = forward(g, r, from, cnt);
+        csd_status s = forward(g, r, from, cnt, from + cnt == P + nd);
         if (s != CSD_OK) return s;
         from += cnt;
     }
@@ -86,11 +147,22 @@ static csd_status review(Gen& g, int r, int P, int nd) {
         }
     }
     const float len_r = r == 0 ? 1.f : g.lenience;   // lenience never applies when the target reviews
+    volatile int32_t* res = g.pinned;
+    res[0] = -1; res[1] = -1;                        // the kernels overwrite both with values >= 0
     csd_status s = csd_spec_accept(target, dl, onehot, g.seq + P, 1, nd, V, g.temperature, len_r, g.seed, g.step++,
                                    g.result_map, g.result_map + 1, g.accept_ws, g.accept_bytes, g.stream);
     if (s != CSD_OK) return s;
-    // the accept kernels write (n_acc, out token) straight into mapped pinned host memory: no copy to wait for
-    CSD_CUDA(cudaStreamSynchronize(g.stream));
+    // The accept kernels write (n_acc, out token) straight into mapped pinned host memory.  The host
+    // watches the two words instead of sleeping in a stream synchronisation (whose wake-up costs more
+    // than the accept call itself) and asks the stream now and then whether it ended early.
+    for (unsigned spins = 0; res[0] < 0 || res[1] < 0; ++spins) {
+        if ((spins & 0x3ff) == 0x3ff) {
+            const cudaError_t q = cudaStreamQuery(g.stream);
+            if (q == cudaSuccess) break;             // stream drained: the words are final
+            if (q != cudaErrorNotReady) return note_cuda(q);
+        }
+    }
+    if (res[0] < 0 || res[1] < 0) CSD_CUDA(cudaStreamSynchronize(g.stream));
     const int n_acc = g.pinned[0];
     if (n_acc < 0 || n_acc > nd) return CSD_ERR_CUDA;
     g.pinned[CSD_MAX_ROWS + 8] = g.pinned[1];     // (a slot the next review does not overwrite while this copy is in flight)
@@ -201,17 +273,16 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
     g.accept_ws = ws + w.accept; g.accept_bytes = w.total - w.accept;
     g.src.assign((size_t)g.cap + 64, 0);
 
-    CSD_CUDA(cudaHostAlloc((void**)&g.pinned, (size_t)(2 + CSD_MAX_ROWS + 64) * 4, cudaHostAllocMapped));
-    if (cudaHostGetDevicePointer((void**)&g.result_map, g.pinned, 0) != cudaSuccess || !g.result_map) {
-        cudaFreeHost(g.pinned);
-        return note_cuda(cudaGetLastError());
+    HostKit kit;
+    {
+        const csd_status ks = kit_acquire(kit);
+        if (ks != CSD_OK) return ks;
     }
-    cudaEvent_t ev0 = nullptr, ev1 = nullptr, ev2 = nullptr;
+    g.pinned = kit.pinned; g.result_map = kit.mapped;
+    cudaEvent_t ev0 = kit.ev[0], ev1 = kit.ev[1], ev2 = kit.ev[2];
     csd_status rc = CSD_OK;
     auto fail = [&](csd_status s) { rc = s; };
     do {
-        if (cudaEventCreate(&ev0) != cudaSuccess || cudaEventCreate(&ev1) != cudaSuccess ||
-            cudaEventCreate(&ev2) != cudaSuccess) { fail(note_cuda(cudaGetLastError())); break; }
         cudaError_t e = cudaMemcpyAsync(g.seq, init_seq_host, (size_t)init_len * 4, cudaMemcpyHostToDevice, g.stream);
         if (e == cudaSuccess && haystack_len > 0)
             e = cudaMemcpyAsync(hay_dev, haystack_host, (size_t)haystack_len * 4, cudaMemcpyHostToDevice, g.stream);
@@ -228,7 +299,7 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
                 int cnt = init_len - 1 - from;
                 const int rows = models[r]->cfg.max_rows < CSD_MAX_ROWS ? models[r]->cfg.max_rows : CSD_MAX_ROWS;
                 if (cnt > rows) cnt = rows;
-                rc = forward(g, r, from, cnt);
+                rc = forward(g, r, from, cnt, false);
                 from += cnt;
             }
             g.kv[r] = init_len - 1;
@@ -256,10 +327,7 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
     } while (0);
     if (rc != CSD_OK) cudaStreamSynchronize(g.stream);
     if (g.mag) csd_mag_destroy(g.mag);
-    if (ev0) cudaEventDestroy(ev0);
-    if (ev1) cudaEventDestroy(ev1);
-    if (ev2) cudaEventDestroy(ev2);
-    cudaFreeHost(g.pinned);
+    kit_release(kit);
     st->kernel_launches = launches_so_far() - launches0;
     st->total_ms = std::chrono::duration<double, std::milli>(std::chrono::steady_clock::now() - t_begin).count();
     return rc;

@@ -462,7 +462,7 @@ extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_token
 
 extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
                                          float* logits_out_dev, void* stream) {
-    if (!M || !block_tokens_dev || !logits_out_dev) return CSD_ERR_INVALID_ARG;
+    if (!M || !block_tokens_dev) return CSD_ERR_INVALID_ARG;
     const csd_model_config& c = M->cfg;
     if (m < 1 || m > c.max_rows || kv_len < 0) return CSD_ERR_INVALID_ARG;
     if (kv_len + m > c.max_seq) return CSD_ERR_CAPACITY;
@@ -530,6 +530,10 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         const bool fused_qkv = nx && nx->wk == nx->wq + (size_t)di * d && nx->wv == nx->wk + (size_t)di * d;
         const int next_N = last ? V : (fused_qkv ? 3 * di : di);
         CSD_TRY(feed_forward(M, y, M->x, m, st, x_ready, next_gain, next_N, false, &x_ready));
+    }
+    if (!logits_out_dev) {                    // cache append only: nobody reads this block's laws
+        CSD_CUDA(cudaGetLastError());
+        return CSD_OK;
     }
     LinOpt ho;
     if (x_ready) { ho.xs_in = M->xs_x; ho.ssq_in = M->ssq_x; ho.ssq_cnt = M->ssq_x_cnt; }
