@@ -277,6 +277,19 @@ def run_ours(args):
         cpu = {"value": n_tok / dt, "unit": "tokens/s", "cores": len(os.sched_getaffinity(0)), "kind": "oracle",
                "sample": f"{ORACLE_PROMPT}-token prompt, {ORACLE_NEW} new tokens, same models and cascade ({dt:.1f} s)"}
 
+    # a short sample of every other configuration, so that each has a figure in this line
+    other = None
+    if world == 1 and not args.no_configs:
+        draft.close()
+        other = {"tiny_cascade": cfg_tiny(b),
+                 "accept": [cfg_accept(b, peak, 128256, 16, 0.5), cfg_accept(b, peak, 128256, 4, 0.5),
+                            cfg_accept(b, peak, 32000, 4, 0.5)],
+                 "long_cache_review_step": cfg_long(b, peak, tb, reviews=6)}
+        target.close()
+        del casc, tb, db
+        torch.cuda.empty_cache()
+        other["t5xxl_target"] = cfg_t5(b, cascade=False)
+
     line = {"metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_per_step, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
@@ -293,7 +306,7 @@ def run_ours(args):
             "review_frac_of_measured": review_gbs / peak,
             "review_split_us": {"gemm": 1e3 * prof["gemm_ms"] / n_rev, "attention": 1e3 * prof["attn_ms"] / n_rev,
                                 "other": 1e3 * prof["other_ms"] / n_rev},
-            "accept_us": accept_us, "kernel_rooflines": kernel_rooflines, "cascade_stats": {k: st[k] for k in ("reviews", "forwards", "drafted", "accepted",
+            "accept_us": accept_us, "kernel_rooflines": kernel_rooflines, "configs": other, "cascade_stats": {k: st[k] for k in ("reviews", "forwards", "drafted", "accepted",
                                                                         "mag_calls")}}
     print(json.dumps(line), flush=True)
     if world > 1:
@@ -333,93 +346,130 @@ def run_review_only(args):
                       "n_acc": int(n_acc[0]), "out": int(out[0])}), flush=True)
 
 
-def run_configs(args):
-    """`--configs a,b,..` measures the other workload configurations (tiny cascade, accept sweep, T5-shaped
-    horizontal cascade, long-cache review) and prints one JSON line each; the default bench line is configuration 3."""
+def timed_us(fn, n):
+    """Mean microseconds per call of fn(i), CUDA events on the current stream."""
+    import torch
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    torch.cuda.synchronize()
+    e0.record()
+    for i in range(n):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return 1e3 * e0.elapsed_time(e1) / n
+
+
+def cfg_tiny(b):
+    """Configuration 1: the tiny cascade (prompt 32, 64 new tokens, greedy, k = 4)."""
     import torch
     import workloads
-    from paper_2312_11462_b200 import binding as b
-    peak, _ = measured_peaks()
-    which = set(args.configs.split(","))
+    ts, ds = workloads.SHAPES["tiny_target"], workloads.SHAPES["tiny_draft"]
+    tb, db = workloads.make_weights(ts, 0, "cuda"), workloads.make_weights(ds, 1, "cuda")
+    prompt = workloads.make_prompt(ts.vocab, 32, seed=0)
+    nxt = torch.from_numpy(workloads.bigram_table(prompt, ts.vocab, seed=0)).cuda()
+    casc = b.Cascade([b.Model(ts, tb), b.Model(ds, db)], K_MATRIX, MAX_BLOCK, nxt, 32)
+    for _ in range(3):
+        casc.csd_cascade_generate(prompt, prompt, 64)
+    t0 = time.time()
+    for _ in range(10):
+        toks, st = casc.csd_cascade_generate(prompt, prompt, 64)
+    dt = (time.time() - t0) / 10
+    return {"config": "1 tiny cascade (prompt 32, 64 new, greedy, k=4)", "tokens_per_s": 64 / dt,
+            "target_forwards_per_token": st["forwards"][0] / 64, "ms_per_generation": 1e3 * dt}
 
-    def timed(fn, n):
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        torch.cuda.synchronize()
-        e0.record()
-        for i in range(n):
-            fn(i)
-        e1.record()
-        torch.cuda.synchronize()
-        return 1e3 * e0.elapsed_time(e1) / n          # microseconds per call
 
-    if "tiny" in which:
-        ts, ds = workloads.SHAPES["tiny_target"], workloads.SHAPES["tiny_draft"]
-        tb, db = workloads.make_weights(ts, 0, "cuda"), workloads.make_weights(ds, 1, "cuda")
-        prompt = workloads.make_prompt(ts.vocab, 32, seed=0)
-        nxt = torch.from_numpy(workloads.bigram_table(prompt, ts.vocab, seed=0)).cuda()
-        casc = b.Cascade([b.Model(ts, tb), b.Model(ds, db)], K_MATRIX, MAX_BLOCK, nxt, 32)
-        for _ in range(3):
-            casc.csd_cascade_generate(prompt, prompt, 64)
-        t0 = time.time()
-        for _ in range(10):
-            toks, st = casc.csd_cascade_generate(prompt, prompt, 64)
-        dt = (time.time() - t0) / 10
-        print(json.dumps({"config": "1 tiny cascade (prompt 32, 64 new, greedy, k=4)", "tokens_per_s": 64 / dt,
-                          "target_forwards_per_token": st["forwards"][0] / 64, "ms_per_generation": 1e3 * dt}), flush=True)
+def cfg_accept(b, peak, V, k, sigma, rows=64):
+    """Configuration 2: one point of the stand-alone accept sweep (fp32 logits, temperature 1)."""
+    import torch
+    import workloads
+    # two input sets, alternated, so that a call never finds its own logits in L2 when they fit
+    sets = [workloads.accept_case(rows, k, V, sigma, seed=7 + j, device="cuda") for j in range(2)]
+    ws = b.csd_spec_accept_workspace(rows, k, V, "cuda")
+    outs = (torch.empty(rows, dtype=torch.int32, device="cuda"), torch.empty(rows, dtype=torch.int32, device="cuda"))
 
-    if "accept" in which:
-        rows = 64
-        for V in (4096, 32000, 128256):
-            for k in (1, 2, 4, 8, 16):
-                for sigma in ((0.1, 0.5, 2.0) if (V, k) == (32000, 4) else (0.5,)):
-                    # two input sets, alternated, so that a call never finds its own logits in L2 when they fit
-                    sets = [workloads.accept_case(rows, k, V, sigma, seed=7 + j, device="cuda") for j in range(2)]
-                    ws = b.csd_spec_accept_workspace(rows, k, V, "cuda")
-                    outs = (torch.empty(rows, dtype=torch.int32, device="cuda"),
-                            torch.empty(rows, dtype=torch.int32, device="cuda"))
+    def call(i):
+        t, d, tok = sets[i & 1]
+        b.csd_spec_accept(t, d, tok, 1.0, seed=11, step=i, workspace=ws, out=outs)
+    for i in range(4):
+        call(i)
+    us = timed_us(call, 20)
+    nbytes = 4.0 * V * (2 * k + 1) * rows
+    return {"config": "2 accept sweep", "V": V, "k": k, "sigma": sigma, "rows": rows, "us": us,
+            "algorithmic_MB": nbytes / 1e6, "GBps": nbytes / us / 1e3, "frac_of_8TBps": nbytes / us / 1e3 / 8000.0,
+            "frac_of_measured": nbytes / us / 1e3 / peak, "mean_accepted": float(outs[0].float().mean())}
 
-                    def call(i):
-                        t, d, tok = sets[i & 1]
-                        b.csd_spec_accept(t, d, tok, 1.0, seed=11, step=i, workspace=ws, out=outs)
-                    for i in range(4):
-                        call(i)
-                    us = timed(call, 20)
-                    nbytes = 4.0 * V * (2 * k + 1) * rows
-                    print(json.dumps({"config": "2 accept sweep", "V": V, "k": k, "sigma": sigma, "rows": rows,
-                                      "us": us, "algorithmic_MB": nbytes / 1e6, "GBps": nbytes / us / 1e3,
-                                      "frac_of_8TBps": nbytes / us / 1e3 / 8000.0,
-                                      "frac_of_measured": nbytes / us / 1e3 / peak,
-                                      "mean_accepted": float(outs[0].float().mean())}), flush=True)
-                    del sets, ws
 
-    if "long" in which:
-        ts = workloads.SHAPES["llama7b_long"]
-        tb = workloads.make_weights(ts, seed=100, device="cuda")
-        target = b.Model(ts, tb)
-        S = 2048
-        prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, S + 17, seed=5)).cuda()
-        for p0 in range(0, S, 16):
-            target.csd_review_forward(prompt[p0:p0 + 16], p0)
-        wbytes = 2.0 * (sum(int(np.prod(sh)) for n, _, sh in workloads.blob_layout(ts)[0]
-                            if "norm" not in n and n != "embed"))
-        for m in (2, 5, 9, 17):
-            blk = prompt[S:S + m].contiguous()
-            logits = torch.empty(m, ts.vocab, device="cuda")
-            for _ in range(3):
-                target.csd_review_forward(blk, S, logits)
-            us = timed(lambda i: target.csd_review_forward(blk, S, logits), 20)
-            kv = 2.0 * 2 * ts.n_layers * ts.d_inner * (S + m)
-            print(json.dumps({"config": "5 long-cache review", "S": S, "m": m, "review_us": us,
-                              "GBps": (wbytes + kv) / us / 1e3, "frac_of_8TBps": (wbytes + kv) / us / 1e3 / 8000.0,
-                              "frac_of_measured": (wbytes + kv) / us / 1e3 / peak}), flush=True)
-        target.close()
-        del tb
+def cfg_long(b, peak, tb, block_rows=(2, 5, 9, 17), reviews=8, S=2048):
+    """Configuration 5: review step (forward + accept) of the 7B-shaped target over a 2048-token cache.
+    The drafted block comes from a stand-in draft whose logits are the target's own along the draft's
+    path plus N(0, 0.5): the harness advances the target one token at a time (untimed) to get those
+    logits, samples the drafts from them, rolls the cache length back and times the review forward and
+    the accept call on the block (temperature 1).  `reviews` consecutive review steps per block size,
+    each continuing from what the previous one accepted."""
+    import torch
+    import workloads
+    ts = workloads.SHAPES["llama7b_long"]
+    target = b.Model(ts, tb)
+    prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, S, seed=5)).cuda()
+    for p0 in range(0, S - 1, 16):
+        target.csd_review_forward(prompt[p0:min(p0 + 16, S - 1)].contiguous(), p0, append_only=True)
+    wbytes = 2.0 * (sum(int(np.prod(sh)) for n, _, sh in workloads.blob_layout(ts)[0] if "norm" not in n and n != "embed"))
+    gen = torch.Generator(device="cuda")
+    gen.manual_seed(55)
+    out = []
+    for m in block_rows:
+        k = m - 1
+        ws = b.csd_spec_accept_workspace(1, k, ts.vocab, "cuda")
+        res = (torch.empty(1, dtype=torch.int32, device="cuda"), torch.empty(1, dtype=torch.int32, device="cuda"))
+        logits = torch.empty(m, ts.vocab, device="cuda")
+        one = torch.empty(1, ts.vocab, device="cuda")
+        pos, last = S - 1, prompt[S - 1:S].clone()          # `last` is the newest token, not yet in the cache
+        us_f, us_a, acc = [], [], []
+        for it in range(reviews + 1):
+            # the stand-in draft's path (untimed): k single-row target forwards
+            toks, dl, cur = [], [], last
+            for i in range(k):
+                target.csd_review_forward(cur.contiguous(), pos + i, one)
+                d = one + 0.5 * torch.randn(one.shape, generator=gen, device="cuda")
+                cur = torch.multinomial(torch.softmax(d.double(), -1), 1, generator=gen).reshape(1).to(torch.int32)
+                toks.append(cur); dl.append(d)
+            block = torch.cat([last] + toks).contiguous()
+            dlog = torch.cat(dl).reshape(1, k, ts.vocab).contiguous()
+            dtok = torch.cat(toks).reshape(1, k).contiguous()
+            e = [torch.cuda.Event(enable_timing=True) for _ in range(3)]
+            torch.cuda.synchronize()
+            e[0].record()
+            target.csd_review_forward(block, pos, logits)                 # rolled back: the block is reviewed at once
+            e[1].record()
+            b.csd_spec_accept(logits.reshape(1, m, ts.vocab), dlog, dtok, 1.0, seed=9, step=it, workspace=ws, out=res)
+            e[2].record()
+            torch.cuda.synchronize()
+            n_acc, tok = int(res[0][0]), int(res[1][0])
+            if it > 0:                                                    # the first step warms up
+                us_f.append(1e3 * e[0].elapsed_time(e[1])); us_a.append(1e3 * e[1].elapsed_time(e[2])); acc.append(n_acc)
+            pos += n_acc + 1
+            last = torch.tensor([tok], dtype=torch.int32, device="cuda")
+        fwd, accept = statistics.median(us_f), statistics.median(us_a)
+        kv = 2.0 * 2 * ts.n_layers * ts.d_inner * (S + m)
+        nbytes = wbytes + kv + 4.0 * ts.vocab * (2 * k + 1)
+        out.append({"config": "5 long-cache review step", "S": S, "m": m, "review_forward_us": fwd, "accept_us": accept,
+                    "step_us": fwd + accept, "mean_accepted": sum(acc) / len(acc), "reviews": len(acc),
+                    "GBps": nbytes / (fwd + accept) / 1e3, "frac_of_8TBps": nbytes / (fwd + accept) / 1e3 / 8000.0,
+                    "frac_of_measured": nbytes / (fwd + accept) / 1e3 / peak})
+    target.close()
+    return out
 
-    if "t5" in which:
-        shapes = [workloads.SHAPES[n] for n in ("t5xxl", "t5base", "t5small")]
-        blobs = [workloads.make_weights(sh, seed=200 + i, device="cuda") for i, sh in enumerate(shapes)]
-        models = [b.Model(sh, w) for sh, w in zip(shapes, blobs)]
-        enc = workloads.make_prompt(shapes[0].vocab, 256, seed=9)
+
+def cfg_t5(b, cascade=True):
+    """Configuration 4: T5-xxl-shaped target with base- and small-shaped drafts, temperature 1."""
+    import torch
+    import workloads
+    shapes = [workloads.SHAPES[n] for n in (("t5xxl", "t5base", "t5small") if cascade else ("t5xxl",))]
+    blobs = [workloads.make_weights(sh, seed=200 + i, device="cuda") for i, sh in enumerate(shapes)]
+    models = [b.Model(sh, w) for sh, w in zip(shapes, blobs)]
+    enc = workloads.make_prompt(shapes[0].vocab, 256, seed=9)
+    res = {"config": "4 T5-xxl-shaped target (encoder 256 tokens)"}
+    if cascade:
         nxt = torch.from_numpy(workloads.bigram_table(enc, shapes[0].vocab, seed=3)).cuda()
         K = [[2, 2, 0], [0, 1, 4], [0, 0, 4]]
         casc = b.Cascade(models, K, 4, nxt, 256)
@@ -428,13 +478,49 @@ def run_configs(args):
         t0 = time.time()
         toks, st = casc.csd_cascade_generate(enc, start, 128, temperature=1.0, seed=2)
         dt = time.time() - t0
-        blk = torch.zeros(5, dtype=torch.int32, device="cuda")
-        logits = torch.empty(5, shapes[0].vocab, device="cuda")
-        us = timed(lambda i: models[0].csd_review_forward(blk, 64, logits), 10)
-        print(json.dumps({"config": "4 T5-xxl-shaped horizontal cascade (encoder 256, 128 new, T=1)",
-                          "tokens_per_s": len(toks) / dt, "prefill_ms": st["prefill_ms"], "decode_ms": st["decode_ms"],
-                          "target_forwards_per_token": st["forwards"][0] / max(len(toks), 1),
-                          "target_review_us_m5": us, "reviews": st["reviews"], "accepted": st["accepted"]}), flush=True)
+        res.update({"cascade": "horizontal [[2,2,0],[0,1,4],[0,0,4]], 128 new, T=1", "tokens_per_s": len(toks) / dt,
+                    "prefill_ms": st["prefill_ms"], "decode_ms": st["decode_ms"],
+                    "target_forwards_per_token": st["forwards"][0] / max(len(toks), 1), "reviews": st["reviews"],
+                    "accepted": st["accepted"]})
+    else:
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        models[0].csd_encoder_forward(torch.from_numpy(enc).cuda())
+        e1.record()
+        torch.cuda.synchronize()
+        res["encoder_ms"] = e0.elapsed_time(e1)
+    blk = torch.zeros(5, dtype=torch.int32, device="cuda")
+    logits = torch.empty(5, shapes[0].vocab, device="cuda")
+    for _ in range(2):
+        models[0].csd_review_forward(blk, 64, logits)
+    res["target_review_us_m5"] = timed_us(lambda i: models[0].csd_review_forward(blk, 64, logits), 10)
+    for m_ in models:
+        m_.close()
+    return res
+
+
+def run_configs(args):
+    """`--configs a,b,..` measures the other workload configurations in full (tiny cascade, accept sweep,
+    T5-shaped horizontal cascade, long-cache review steps) and prints one JSON line each; the default
+    bench line is configuration 3 and carries a short sample of each of them."""
+    import workloads
+    from paper_2312_11462_b200 import binding as b
+    peak, _ = measured_peaks()
+    which = set(args.configs.split(","))
+    if "tiny" in which:
+        print(json.dumps(cfg_tiny(b)), flush=True)
+    if "accept" in which:
+        for V in (4096, 32000, 128256):
+            for k in (1, 2, 4, 8, 16):
+                for sigma in ((0.1, 0.5, 2.0) if (V, k) == (32000, 4) else (0.5,)):
+                    print(json.dumps(cfg_accept(b, peak, V, k, sigma)), flush=True)
+    if "long" in which:
+        tb = workloads.make_weights(workloads.SHAPES["llama7b_long"], seed=100, device="cuda")
+        for line in cfg_long(b, peak, tb, reviews=32):
+            print(json.dumps(line), flush=True)
+        del tb
+    if "t5" in which:
+        print(json.dumps(cfg_t5(b, cascade=True)), flush=True)
 
 
 def main():
@@ -444,6 +530,7 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-configs", action="store_true", help="leave the samples of the other configurations out of the line")
     ap.add_argument("--review-only", type=int, default=0, help="profiling aid: only N review forwards of the target")
     ap.add_argument("--layers", type=int, default=0, help="with --review-only: cut the target to L layers")
     ap.add_argument("--configs", default="", help="measure other configurations: tiny,accept,long,t5")

@@ -11,10 +11,11 @@ from gpu_util import LOGIT_MAX_ABS, LOGIT_REL_L2, rel_l2, require_gpu, to_dev_i3
 pytestmark = pytest.mark.gpu
 
 
-@pytest.fixture(scope="module", params=[1, 2, 3], ids=["cuda-core", "tensor-core", "tensor-core-row-ranges"])
+@pytest.fixture(scope="module", params=[0, 1, 2, 3], ids=["automatic", "cuda-core", "tensor-core", "tensor-core-row-ranges"])
 def b(request):
-    """Every test here runs once per kernel family: CUDA-core GEMM (128-bit loads + fp32 FMA) with the
-    CUDA-core attention, and tensor-core GEMM (TMA + tcgen05) with the tensor-core attention."""
+    """Every test here runs once per kernel family: the automatic choice (small models go through the
+    whole-forward kernel), CUDA-core GEMM (128-bit loads + fp32 FMA) with the CUDA-core attention, and
+    the two tensor-core GEMMs (TMA + tcgen05) with the tensor-core attention."""
     require_gpu()
     from paper_2312_11462_b200 import binding
     binding.csd_set_gemm_path(request.param)
