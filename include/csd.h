@@ -231,6 +231,13 @@ csd_status csd_mag_destroy(csd_mag* g);
 /* seq_dev [T] (T >= 1), 1 <= n <= 64; writes out_tokens_dev [n] (may alias seq_dev + T). */
 csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32_t* out_tokens_dev,
                          void* stream);
+/* The same search over a haystack that grows with the generation (Section 3.3 takes the match from
+ * the input or from the existing generation): the handle's haystack followed by
+ * seq_dev[gen_from .. T), 0 <= gen_from <= T.  A match must still be followed by a token of that
+ * joined text, and the earliest occurrence wins, so the static part is preferred.  The generated
+ * part is scanned directly on every call: it may shrink when a block is rejected. */
+csd_status csd_mag_draft_dynamic(csd_mag* g, const int32_t* seq_dev, int T, int gen_from, int n,
+                                 int32_t* out_tokens_dev, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Algorithm 1 (CascadeSpeculativeDraftingStep) driven until max_new tokens exist.
@@ -244,6 +251,8 @@ csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32
  * cached yet, in chunks of at most the model's max_rows rows (this also serves as prompt prefill).
  * Decoder-only models: haystack = prompt, init_seq = prompt.  Encoder-decoder: haystack =
  * encoder input (the encoders are run here), init_seq = decoder start token(s).
+ * dynamic_haystack != 0: Max-Gram also matches inside everything generated so far (the tokens after
+ * init_seq, drafts that are still under review included), see csd_mag_draft_dynamic.
  * Host in, host out; the call returns after the stream has finished.
  * ------------------------------------------------------------------------------------------- */
 typedef struct {
@@ -263,7 +272,7 @@ typedef struct {
 size_t csd_cascade_workspace_bytes(int vocab, int max_block, int seq_capacity, int haystack_len, int max_order);
 csd_status csd_cascade_generate(csd_model* const* models, int n_levels, const int32_t* K, int max_block,
                                 float lenience, float temperature, uint64_t seed, int max_order,
-                                const int32_t* haystack_host, int haystack_len,
+                                int dynamic_haystack, const int32_t* haystack_host, int haystack_len,
                                 const int32_t* bigram_next_dev, const int32_t* init_seq_host, int init_len,
                                 int max_new, int32_t* out_tokens_host, int32_t* out_len,
                                 csd_cascade_stats* stats,

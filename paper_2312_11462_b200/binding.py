@@ -93,9 +93,10 @@ lib.csd_mag_workspace_bytes.argtypes = [_i, _i, _i]
 lib.csd_mag_create.argtypes = [_vp, _i, _i, _vp, _i, _i, _vp, _sz, _vp, _vp]
 lib.csd_mag_destroy.argtypes = [_vp]
 lib.csd_mag_draft.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
+lib.csd_mag_draft_dynamic.argtypes = [_vp, _vp, _i, _i, _i, _vp, _vp]
 lib.csd_cascade_workspace_bytes.restype = _sz
 lib.csd_cascade_workspace_bytes.argtypes = [_i, _i, _i, _i, _i]
-lib.csd_cascade_generate.argtypes = [_vp, _i, _vp, _i, _f, _f, _u64, _i, _vp, _i, _vp, _vp, _i, _i, _vp, _vp, _vp,
+lib.csd_cascade_generate.argtypes = [_vp, _i, _vp, _i, _f, _f, _u64, _i, _i, _vp, _i, _vp, _vp, _i, _i, _vp, _vp, _vp,
                                      _vp, _sz, _vp]
 lib.csd_rel_bucket.argtypes = [_i, _i, _i, _i]
 
@@ -282,6 +283,14 @@ class Mag:
         _check("csd_mag_draft", lib.csd_mag_draft(self.h, _ptr(seq), seq.numel(), n, _ptr(out), _stream()))
         return out
 
+    def csd_mag_draft_dynamic(self, seq: torch.Tensor, gen_from: int, n: int) -> torch.Tensor:
+        """Haystack = the handle's haystack followed by seq[gen_from:]."""
+        assert seq.dtype == torch.int32 and seq.is_cuda and seq.is_contiguous()
+        out = torch.empty(n, dtype=torch.int32, device=seq.device)
+        _check("csd_mag_draft_dynamic",
+               lib.csd_mag_draft_dynamic(self.h, _ptr(seq), seq.numel(), gen_from, n, _ptr(out), _stream()))
+        return out
+
     def close(self) -> None:
         if getattr(self, "h", None):
             lib.csd_mag_destroy(self.h)
@@ -314,7 +323,8 @@ class Cascade:
         self.handles = (C.c_void_p * n)(*[m.h for m in self.models])
 
     def csd_cascade_generate(self, haystack: np.ndarray, init_seq: np.ndarray, max_new: int,
-                             temperature: float = 0.0, lenience: float = 1.0, seed: int = 0):
+                             temperature: float = 0.0, lenience: float = 1.0, seed: int = 0,
+                             dynamic_haystack: bool = False):
         """Host in, host out.  Returns (tokens int32 numpy, stats dict)."""
         hay = np.ascontiguousarray(haystack, dtype=np.int32)
         init = np.ascontiguousarray(init_seq, dtype=np.int32)
@@ -323,7 +333,8 @@ class Cascade:
         out_len = C.c_int32(0)
         st = CascadeStats()
         code = lib.csd_cascade_generate(self.handles, len(self.models), self.K.ctypes.data_as(_vp), self.max_block,
-                                        lenience, temperature, seed, self.max_order, hay.ctypes.data_as(_vp),
+                                        lenience, temperature, seed, self.max_order, int(dynamic_haystack),
+                                        hay.ctypes.data_as(_vp),
                                         len(hay), _ptr(self.bigram), init.ctypes.data_as(_vp), len(init), max_new,
                                         out.ctypes.data_as(_vp), C.byref(out_len), C.byref(st), _ptr(self.workspace),
                                         self.workspace.numel(), _stream())

@@ -94,7 +94,7 @@ static void kit_release(HostKit& k) {
 
 struct Gen {
     csd_model* const* models; int n_levels; const int32_t* K; int max_block; float lenience, temperature;
-    uint64_t seed, step = 0; csd_mag* mag = nullptr; int V, cap;
+    uint64_t seed, step = 0; csd_mag* mag = nullptr; int V, cap; int dynamic = 0, init_len = 0;
     int32_t* seq; int len = 0; int kv[8] = {0};
     std::vector<signed char> src;        // per position: proposing level, -1 = point mass
     float *law, *qlaw, *dl; int32_t *onehot_dev, *result_dev, *result_map = nullptr; void* accept_ws; size_t accept_bytes;
@@ -187,7 +187,8 @@ static csd_status step(Gen& g, int r, int budget) {
     if (r == g.n_levels) {   // base case: the statistical drafter proposes the slot's remaining budget
         if (budget < 1) budget = 1;
         if (g.len + budget > g.cap) return CSD_ERR_CAPACITY;
-        csd_status s = csd_mag_draft(g.mag, g.seq, g.len, budget, g.seq + g.len, g.stream);
+        csd_status s = g.dynamic ? csd_mag_draft_dynamic(g.mag, g.seq, g.len, g.init_len, budget, g.seq + g.len, g.stream)
+                                 : csd_mag_draft(g.mag, g.seq, g.len, budget, g.seq + g.len, g.stream);
         if (s != CSD_OK) return s;
         for (int i = 0; i < budget; ++i) g.src[g.len + i] = -1;
         g.len += budget;
@@ -227,7 +228,7 @@ extern "C" size_t csd_cascade_workspace_bytes(int vocab, int max_block, int seq_
 
 extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_levels, const int32_t* K, int max_block,
                                            float lenience, float temperature, uint64_t seed, int max_order,
-                                           const int32_t* haystack_host, int haystack_len,
+                                           int dynamic_haystack, const int32_t* haystack_host, int haystack_len,
                                            const int32_t* bigram_next_dev, const int32_t* init_seq_host, int init_len,
                                            int max_new, int32_t* out_tokens_host, int32_t* out_len,
                                            csd_cascade_stats* stats, void* workspace_dev, size_t workspace_bytes,
@@ -253,6 +254,7 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
     g.models = models; g.n_levels = n_levels; g.K = K; g.max_block = max_block; g.lenience = lenience;
     g.temperature = temperature; g.seed = seed; g.V = models[0]->cfg.vocab; g.st = st;
     g.stream = (cudaStream_t)stream;
+    g.dynamic = dynamic_haystack != 0; g.init_len = init_len;
     g.cap = models[0]->cfg.max_seq;
     for (int r = 1; r < n_levels; ++r)
         if (models[r]->cfg.max_seq < g.cap) g.cap = models[r]->cfg.max_seq;

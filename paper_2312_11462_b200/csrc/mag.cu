@@ -7,6 +7,15 @@
 // Draft: one warp; lane o-1 probes the table for the suffix of order o, the longest hit wins
 // (a suffix of order o that matches implies every shorter one matches), then the tokens after
 // the hit are copied; without a hit one token comes from the bigram table.
+//
+// Dynamic haystack (Section 3.3 lets the match come from the input or from the existing
+// generation): the haystack is the static one followed by the generated part of the sequence,
+// seq[gen_from, T).  The table still covers every occurrence that ends at least two tokens before
+// the end of the static part; occurrences that end later (their follower, or part of them, is
+// generated text, which comes and goes as blocks are rejected) are few and are found by a direct
+// scan: every lane takes candidate end positions in turn, counts how far the text before them
+// agrees with the sequence's tail, and records the earliest end per order.  Table hits start
+// earlier than scanned ones by construction, so per order the table wins when it has a hit.
 #include "common.cuh"
 
 struct csd_mag {
@@ -70,8 +79,12 @@ constexpr int MAG_MAX_N = 64;
 
 __global__ void __launch_bounds__(32)
 mag_draft_kernel(const int32_t* __restrict__ hay, int L, const int32_t* __restrict__ bigram, int V,
-                 const int* __restrict__ table, int slots, int max_order, const int32_t* __restrict__ seq, int T,
-                 int n, int32_t* __restrict__ out, int* status) {
+                 const int* __restrict__ table, int slots, int max_order, const int32_t* seq, int T,
+                 int gen_from, int n, int32_t* out, int* status) {
+    // joined haystack: hay[0, L) followed by seq[gen_from, T) when gen_from >= 0
+    const int G = gen_from >= 0 ? T - gen_from : 0, LJ = L + G;
+    auto joined = [&](int i) { return i < L ? hay[i] : seq[gen_from + (i - L)]; };
+    __shared__ int best_end[CSD_MAG_MAX_ORDER + 1];
     // tail = last max_order tokens of the sequence followed by the tokens proposed so far
     // (at most CSD_MAG_MAX_ORDER + MAG_MAX_N entries, so it never overflows)
     __shared__ int32_t tail[CSD_MAG_MAX_ORDER + MAG_MAX_N];
@@ -96,6 +109,19 @@ mag_draft_kernel(const int32_t* __restrict__ hay, int L, const int32_t* __restri
                 h = (h + 1) & (uint32_t)(slots - 1);
             }
         }
+        if (G > 0) {
+            // ends e in [L-1, LJ-2]: the occurrence's follower e+1 exists and is generated text
+            best_end[lane + 1] = 0x7fffffff;
+            __syncwarp();
+            for (int e = max(L - 1, 0) + lane; e <= LJ - 2; e += 32) {
+                int agree = 0;
+                while (agree < limit && agree <= e && joined(e - agree) == tail[len - 1 - agree]) ++agree;
+                for (int o = 1; o <= agree; ++o) atomicMin(&best_end[o], e);
+            }
+            __syncwarp();
+            if (hit < 0 && order <= limit && best_end[order] != 0x7fffffff) hit = best_end[order] - order + 1;
+            __syncwarp();
+        }
         const unsigned ballot = __ballot_sync(0xffffffffu, hit >= 0);
         if (ballot == 0) {
             int32_t last = tail[len - 1];
@@ -108,9 +134,9 @@ mag_draft_kernel(const int32_t* __restrict__ hay, int L, const int32_t* __restri
             const int best = 31 - __clz(ballot);              // lane of the longest order that hit
             const int start = __shfl_sync(0xffffffffu, hit, best);
             int idx = start + best + 1;                      // haystack index of the next token
-            int cnt = min(n - made, L - idx);
+            int cnt = min(n - made, LJ - idx);
             for (int i = lane; i < cnt; i += 32) {
-                int32_t t = hay[idx + i];
+                int32_t t = joined(idx + i);
                 tail[len + i] = t;
                 out[made + i] = t;
             }
@@ -177,15 +203,26 @@ extern "C" csd_status csd_mag_destroy(csd_mag* g) {
     return CSD_OK;
 }
 
-extern "C" csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32_t* out_tokens_dev,
-                                    void* stream) {
+static csd_status mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int gen_from, int n, int32_t* out_tokens_dev,
+                            void* stream) {
     if (!g || !seq_dev || !out_tokens_dev || T < 1) return CSD_ERR_INVALID_ARG;
     if (n < 1 || n > MAG_MAX_N) return CSD_ERR_INVALID_ARG;
     int* status = status_word_device();
     if (!status) return CSD_ERR_CUDA;
     mag_draft_kernel<<<1, 32, 0, (cudaStream_t)stream>>>(g->hay, g->L, g->bigram, g->V, g->table, g->slots,
-                                                          g->max_order, seq_dev, T, n, out_tokens_dev, status);
+                                                          g->max_order, seq_dev, T, gen_from, n, out_tokens_dev, status);
     count_launch();
     CSD_CUDA(cudaGetLastError());
     return CSD_OK;
+}
+
+extern "C" csd_status csd_mag_draft(csd_mag* g, const int32_t* seq_dev, int T, int n, int32_t* out_tokens_dev,
+                                    void* stream) {
+    return mag_draft(g, seq_dev, T, -1, n, out_tokens_dev, stream);
+}
+
+extern "C" csd_status csd_mag_draft_dynamic(csd_mag* g, const int32_t* seq_dev, int T, int gen_from, int n,
+                                            int32_t* out_tokens_dev, void* stream) {
+    if (gen_from < 0 || gen_from > T) return CSD_ERR_INVALID_ARG;
+    return mag_draft(g, seq_dev, T, gen_from, n, out_tokens_dev, stream);
 }

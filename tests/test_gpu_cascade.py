@@ -113,6 +113,30 @@ def test_accepting_cascade_and_repetitive_prompt(b, orc):
     assert st["accepted"][0] > 0
 
 
+def test_dynamic_haystack_cascade(b, orc):
+    # Max-Gram may match inside the generation (Section 3.3).  A 24-token vocabulary makes the
+    # generated text repeat itself, and a draft equal to the target accepts what the matches propose:
+    # with the dynamic haystack more Max-Gram tokens survive the draft's review than with the static one.
+    from workloads import llama_shape
+    ts = llama_shape(2, 64, 2, 128, 24, 200)
+    tb = workloads.make_weights(ts, seed=3, device="cpu", std=0.6)    # seed with wide margins on all 80 steps
+    prompt = workloads.make_prompt(ts.vocab, 12, seed=3)
+    nxt = workloads.bigram_table(prompt, ts.vocab, seed=0)
+    K = [[3, 3], [0, 6]]
+    accepted = {}
+    for dyn in (False, True):
+        oms = [orc.Model(ts, orc.blob_to_u16(tb)) for _ in range(2)]
+        want, margins, ost = orc.cascade_generate(oms, prompt, nxt, K, 6, prompt, 80, dynamic_haystack=dyn)
+        gms = [b.Model(ts, tb.cuda()), b.Model(ts, tb.cuda())]
+        got, st = b.Cascade(gms, K, 6, to_dev_i32(nxt), 64).csd_cascade_generate(prompt, prompt, 80, dynamic_haystack=dyn)
+        assert agreed_prefix(got, want, margins) == 80
+        assert st["reviews"] == ost["reviews"] and st["accepted"] == ost["accepted"] and st["mag_calls"] == ost["mag_calls"]
+        assert list(got) == gpu_target_only_greedy(b, ts, tb.cuda(), prompt, 80)      # lossless either way
+        accepted[dyn] = st["accepted"][1]
+    assert accepted[True] > accepted[False]
+    assert b.csd_device_status() == 0
+
+
 def test_teacher_forced_logits_follow_the_oracle(b, orc):
     ts = SHAPES["tiny_target"]
     tb = workloads.make_weights(ts, seed=0, device="cuda")

@@ -77,3 +77,36 @@ def test_in_place_append_and_errors(b, orc):
     assert lib.csd_mag_draft(g.h, _ptr(buf), 5, 65, _ptr(buf), _stream()) == 1
     with pytest.raises(b.CsdError):
         b.Mag(to_dev_i32(hay), to_dev_i32(nxt), 16, 64)      # table too small for the n-grams
+
+
+def test_dynamic_haystack_against_the_oracle(b, orc):
+    # haystack = static part followed by the generated part of the sequence; the oracle searches the
+    # joined text.  Small vocabularies and repeated phrases make matches that lie inside the static
+    # part, straddle its end, lie inside the generation, or whose follower is the first generated token.
+    rng = np.random.default_rng(1)
+    for trial in range(150):
+        V = int(rng.choice([3, 5, 50]))
+        L = int(rng.integers(0, 80))
+        P = int(rng.integers(1, 20))                       # tokens of the sequence before the generation
+        G = int(rng.integers(0, 70))                       # generated tokens
+        n = int(rng.integers(1, 17))
+        order = int(rng.choice([1, 2, 3, 16, 32]))
+        hay = (workloads.make_repetitive_prompt(V, L, int(rng.integers(1 << 30))) if trial % 2 == 0 and L > 0
+               else rng.integers(0, V, size=L).astype(np.int32))
+        seq = rng.integers(0, V, size=P + G).astype(np.int32)
+        if trial % 3 == 0 and G > 12:                      # a phrase repeated inside the generation
+            w = int(rng.integers(2, 6))
+            seq[P + G - w:] = seq[P + 2:P + 2 + w]
+        if trial % 3 == 1 and L > 4 and G >= 3:            # the generation continues the static part's end
+            seq[-2:] = hay[-2:]
+        nxt = rng.integers(0, V, size=V).astype(np.int32)
+        joined = np.concatenate([hay, seq[P:]]).astype(np.int32)
+        want = orc.mag_draft(joined, nxt, seq, n, order)
+        g = b.Mag(to_dev_i32(hay) if L > 0 else to_dev_i32([0])[:0], to_dev_i32(nxt), order)
+        got = g.csd_mag_draft_dynamic(to_dev_i32(seq), P, n).cpu().numpy()
+        assert got.tolist() == want.tolist(), (trial, hay, seq, P, n, order)
+        # nothing generated yet: the static search
+        got0 = g.csd_mag_draft_dynamic(to_dev_i32(seq[:P]), P, n).cpu().numpy()
+        assert got0.tolist() == orc.mag_draft(hay, nxt, seq[:P], n, order).tolist()
+        g.close()
+    assert b.csd_device_status() == 0
