@@ -120,6 +120,14 @@ csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int 
 csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
                               float* logits_out_dev, void* stream);
 
+/* Prompt prefill: the model takes the input tokens in one run (Section 2).  Appends n tokens
+ * (any n >= 1 with kv_len + n <= max_seq) at positions kv_len .. kv_len+n-1 to the cache of every
+ * layer and produces no logits.  Models whose layer matrices are large enough for the tensor-core
+ * kernels go through the weights once per 128 tokens (wide blocks, two bf16 terms per fp32
+ * activation); the rest, and a remainder of at most max_rows tokens, go through the review
+ * kernels.  arch 1: decoder tokens, after csd_encoder_forward. */
+csd_status csd_prefill(csd_model* m, const int32_t* tokens_dev, int n, int kv_len, void* stream);
+
 /* Per-kernel-class timing of later forwards of this model (measurement aid; the paper's unit of
  * cost is "a single run" of a model, Section 4).  While enabled, every kernel launch of
  * csd_review_forward is bracketed by a CUDA event pair on the launching stream (a few
@@ -139,7 +147,9 @@ csd_status csd_model_profile_read(csd_model* m, void* stream, csd_profile* out);
 
 /* Y[m, N] = X[m, K] . W[N, K]^T, the weight-streaming contraction every layer of the review
  * forward is made of (W bf16 row-major, X and Y fp32 row-major, fp32 accumulation).  Exposed
- * for kernel-level tests and roofline measurements.  1 <= m <= 17, K multiple of 8. */
+ * for kernel-level tests and roofline measurements.  K multiple of 8; 1 <= m <= 17 runs the review
+ * kernels, 18 <= m <= 128 the wide-block kernel of the prefill (two bf16 terms per fp32 value, relative
+ * error about 1e-5; needs N * K >= 2^20 and K >= 64, CSD_ERR_UNSUPPORTED otherwise). */
 size_t csd_linear_workspace_bytes(int m, int N, int K);
 /* Which kernel the contraction uses, process-wide: 0 = automatic choice per shape, 1 = the
  * CUDA-core kernel (128-bit streaming loads, fp32 FMA), 2 = the tensor-core kernel (TMA-staged

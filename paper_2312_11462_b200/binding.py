@@ -76,6 +76,7 @@ lib.csd_model_create.argtypes = [_vp, _vp, _sz, _vp, _sz, _vp, _vp]
 lib.csd_model_destroy.argtypes = [_vp]
 lib.csd_encoder_forward.argtypes = [_vp, _vp, _i, _vp]
 lib.csd_review_forward.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
+lib.csd_prefill.argtypes = [_vp, _vp, _i, _i, _vp]
 lib.csd_model_profile.argtypes = [_vp, _i]
 lib.csd_model_profile_read.argtypes = [_vp, _vp, _vp]
 lib.csd_set_gemm_path.argtypes = [_i]
@@ -170,6 +171,11 @@ class Model:
         _check("csd_review_forward",
                lib.csd_review_forward(self.h, _ptr(block_tokens), m, kv_len, _ptr(logits_out), _stream()))
         return logits_out
+
+    def csd_prefill(self, tokens: torch.Tensor, kv_len: int) -> None:
+        """Appends the tokens to the cache (wide blocks where the model allows them); no logits."""
+        assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.is_contiguous()
+        _check("csd_prefill", lib.csd_prefill(self.h, _ptr(tokens), tokens.numel(), kv_len, _stream()))
 
     def csd_model_profile(self, enable: bool) -> None:
         _check("csd_model_profile", lib.csd_model_profile(self.h, int(enable)))

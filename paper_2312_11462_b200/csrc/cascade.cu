@@ -297,12 +297,10 @@ extern "C" csd_status csd_cascade_generate(csd_model* const* models, int n_level
         // prefill: encoders (encoder-decoder models), then every prompt token but the last
         for (int r = 0; r < n_levels && rc == CSD_OK; ++r) {
             if (models[r]->cfg.arch == 1) rc = csd_encoder_forward(models[r], hay_dev, haystack_len, g.stream);
-            for (int from = 0; rc == CSD_OK && from < init_len - 1;) {
-                int cnt = init_len - 1 - from;
+            if (rc == CSD_OK && init_len > 1) {
+                rc = csd_prefill(models[r], g.seq, init_len - 1, 0, g.stream);
                 const int rows = models[r]->cfg.max_rows < CSD_MAX_ROWS ? models[r]->cfg.max_rows : CSD_MAX_ROWS;
-                if (cnt > rows) cnt = rows;
-                rc = forward(g, r, from, cnt, false);
-                from += cnt;
+                g.st->forwards[r] += (init_len - 1 + rows - 1) / rows;   // counted in review-sized blocks
             }
             g.kv[r] = init_len - 1;
         }

@@ -400,16 +400,17 @@ struct LinearWs { size_t tickets, partial, xs, ssq, total; };
 static LinearWs linear_ws(int m, int N, int K) {
     LinearWs w;
     size_t off = 0;
+    const int rows = m > CSD_MAX_ROWS ? CSD_WIDE_ROWS : CSD_MAX_ROWS;
     w.tickets = off; off += align_up((size_t)linear_ticket_count(N) * sizeof(unsigned), 256);
-    w.partial = off; off += linear_scratch_bytes(m, N, K, false);
-    w.xs = off;      off += align_up((size_t)3 * CSD_MAX_ROWS * K * 2, 256);
-    w.ssq = off;     off += align_up((size_t)split_ssq_entries(K) * CSD_MAX_ROWS * sizeof(float), 256);
+    w.partial = off; off += linear_scratch_bytes(m > CSD_MAX_ROWS ? CSD_MAX_ROWS : m, N, K, false);
+    w.xs = off;      off += align_up((size_t)3 * rows * K * 2, 256);
+    w.ssq = off;     off += align_up((size_t)split_ssq_entries(K) * rows * sizeof(float), 256);
     w.total = off;
     return w;
 }
 
 extern "C" size_t csd_linear_workspace_bytes(int m, int N, int K) {
-    if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8) return 0;
+    if (m < 1 || m > CSD_WIDE_ROWS || N < 1 || K < 8) return 0;
     return linear_ws(m, N, K).total;
 }
 
@@ -417,12 +418,21 @@ extern "C" size_t csd_linear_workspace_bytes(int m, int N, int K) {
 // leaves the tickets zero again, so one cudaMemset after allocation is enough.
 extern "C" csd_status csd_linear(const void* W_bf16_dev, int N, int K, const float* X_dev, int m, float* Y_dev,
                                  void* workspace_dev, size_t workspace_bytes, void* stream) {
-    if (m < 1 || m > CSD_MAX_ROWS || N < 1 || K < 8 || (K & 7)) return CSD_ERR_INVALID_ARG;
+    if (m < 1 || m > CSD_WIDE_ROWS || N < 1 || K < 8 || (K & 7)) return CSD_ERR_INVALID_ARG;
     if (!W_bf16_dev || !X_dev || !Y_dev || !workspace_dev) return CSD_ERR_INVALID_ARG;
     const LinearWs w = linear_ws(m, N, K);
     if (workspace_bytes < w.total) return CSD_ERR_CAPACITY;
     if (((uintptr_t)workspace_dev) & 255) return CSD_ERR_INVALID_ARG;
     char* ws = (char*)workspace_dev;
+    if (m > CSD_MAX_ROWS) {                  // wide block: two-term rows, the wide tensor-core kernel
+        if (!wide_supported(m, N, K, false)) return CSD_ERR_UNSUPPORTED;
+        csd_status s = launch_wide_split(X_dev, K, K, m, nullptr, (__nv_bfloat16*)(ws + w.xs), nullptr, (cudaStream_t)stream);
+        if (s != CSD_OK) return s;
+        WideArgs wa;
+        wa.W = (const __nv_bfloat16*)W_bf16_dev; wa.N = N; wa.K = K; wa.m = m; wa.xs = (const __nv_bfloat16*)(ws + w.xs);
+        wa.Y = Y_dev; wa.ldy = N; wa.epilogue = EPI_STORE;
+        return launch_linear_wide(wa, (cudaStream_t)stream);
+    }
     LinearArgs a;
     a.W = (const __nv_bfloat16*)W_bf16_dev; a.N = N; a.K = K; a.X = X_dev; a.ldx = K; a.m = m;
     a.Y = Y_dev; a.ldy = N; a.epilogue = EPI_STORE;

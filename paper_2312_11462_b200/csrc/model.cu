@@ -136,9 +136,18 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
-        buckets, gemm_partial, gemm_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x, total;
+        buckets, gemm_partial, gemm_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x,
+        wx, wqkv, wattn, wact, wxs_x, wxs_attn, wxs_act, wssq, total;
+    bool wide;
     size_t layer_kv, layer_x;
 };
+
+// The wide-block path serves a model when each of its layer matrices takes the wide kernel at 128 rows.
+static bool wide_capable(const csd_model_config& c) {
+    const int d = c.d_model, di = c.n_heads * c.d_head, ff = c.d_ff, R = CSD_WIDE_ROWS;
+    return wide_supported(R, di, d, false) && wide_supported(R, 3 * di, d, false) && wide_supported(R, d, di, false) &&
+           wide_supported(R, ff, d, true) && wide_supported(R, d, ff, false);
+}
 
 static WsLayout ws_layout(const csd_model_config& c) {
     WsLayout L{};
@@ -169,6 +178,16 @@ static WsLayout ws_layout(const csd_model_config& c) {
     L.xs_attn = put(3 * R * di * 2);
     L.xs_act = put(3 * R * ff * 2);
     L.ssq_x = put((size_t)linear_ssq_capacity((int)d) * R * 4);
+    L.wide = wide_capable(c);
+    if (L.wide) {
+        const size_t WR = CSD_WIDE_ROWS;
+        L.wx = put(WR * d * 4); L.wqkv = put(WR * 3 * di * 4); L.wattn = put(WR * di * 4); L.wact = put(WR * ff * 4);
+        L.wxs_x = put(2 * WR * d * 2); L.wxs_attn = put(2 * WR * di * 2); L.wxs_act = put(2 * WR * ff * 2);
+        const size_t kmax_w = d > di ? (d > ff ? d : ff) : (di > ff ? di : ff);
+        size_t pieces = (size_t)wide_ssq_capacity((int)d);
+        if ((size_t)wide_split_pieces((int)kmax_w) > pieces) pieces = (size_t)wide_split_pieces((int)kmax_w);
+        L.wssq = put(pieces * WR * 4);
+    }
     if (c.arch == 0) {
         L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
         L.rope_s = put((size_t)c.max_seq * (Dh / 2) * 4);
@@ -280,6 +299,102 @@ static csd_status feed_forward(csd_model* M, const LayerW& y, float* X, int m, c
     return linear(M, y.wdown, nullptr, d, ff, M->act, ff, m, nullptr, X, d, EPI_ADD, st, &down);
 }
 
+// ---------------------------------------------------------------------------------------------
+// wide blocks: one pass of the decoder over up to CSD_WIDE_ROWS rows that only fills the cache
+// ---------------------------------------------------------------------------------------------
+static csd_status wide_linear(csd_model* M, const __nv_bfloat16* W, const __nv_bfloat16* W2, int N, int K, int m,
+                              const __nv_bfloat16* xs, const float* ssq, int ssq_cnt, float* Y, int ldy, int epi,
+                              __nv_bfloat16* out_xs, int out_ld, const __nv_bfloat16* out_gain, float* out_ssq,
+                              cudaStream_t st) {
+    WideArgs a;
+    a.W = W; a.W2 = W2; a.N = N; a.K = K; a.m = m; a.xs = xs; a.ssq = ssq; a.ssq_cnt = ssq_cnt; a.eps = M->cfg.norm_eps;
+    a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.out_xs = out_xs; a.out_ld = out_ld; a.out_gain = out_gain; a.out_ssq = out_ssq;
+    ProfScope ps(M, 0, st);
+    if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
+    return launch_linear_wide(a, st);
+}
+
+// Attention of `m` rows (any number) in sub-blocks of at most CSD_MAX_ROWS over K/V that are already
+// in the cache: row r sees keys [0, n_keys0 + r) when causal, all n_keys0 otherwise.
+static csd_status wide_attention(csd_model* M, const float* q, int ldq, int m, __nv_bfloat16* Kc, __nv_bfloat16* Vc, int cap,
+                                 int n_keys0, bool causal, const float* bias, int bias_len, int bias_zero, int q_pos0,
+                                 float* out, cudaStream_t st) {
+    const csd_model_config& c = M->cfg;
+    for (int r0 = 0; r0 < m; r0 += CSD_MAX_ROWS) {
+        AttnArgs a;
+        a.q = q + (size_t)r0 * ldq; a.ldq = ldq; a.m = m - r0 < CSD_MAX_ROWS ? m - r0 : CSD_MAX_ROWS;
+        a.Kc = Kc; a.Vc = Vc; a.cap = cap; a.H = c.n_heads; a.Dh = c.d_head;
+        a.n_keys = causal ? n_keys0 + r0 : n_keys0; a.causal = causal ? 1 : 0;
+        a.scale = c.arch == 0 ? 1.f / sqrtf((float)c.d_head) : 1.f;
+        a.bias = bias; a.bias_len = bias_len; a.bias_zero = bias_zero; a.q_pos0 = q_pos0 + r0;
+        a.out = out + (size_t)r0 * M->di; a.ldo = M->di;
+        CSD_TRY(attention(M, a, st));
+    }
+    return CSD_OK;
+}
+
+// Decoder pass over m <= CSD_WIDE_ROWS rows at positions kv_len .. kv_len+m-1: K/V of every layer are
+// appended, nothing else is kept.
+static csd_status wide_decoder_pass(csd_model* M, const int32_t* tokens, int m, int kv_len, cudaStream_t st) {
+    const csd_model_config& c = M->cfg;
+    const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, ff = c.d_ff;
+    {
+        ProfScope ps(M, 2, st);
+        embed_kernel<<<m, 128, 0, st>>>(tokens, M->embed, c.vocab, d, M->wx, M->status);
+        count_launch();
+    }
+    int cnt = 0;                       // pieces in wssq that describe the rows in wxs_x (0: wxs_x not current)
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerW& y = M->dec[l];
+        __nv_bfloat16* Kl = M->kcache + (size_t)l * M->layer_kv;
+        __nv_bfloat16* Vl = M->vcache + (size_t)l * M->layer_kv;
+        if (cnt == 0) {
+            CSD_TRY(launch_wide_split(M->wx, d, d, m, y.norm1, M->wxs_x, M->wssq, st));
+            cnt = wide_split_pieces(d);
+        }
+        if (y.wk == y.wq + (size_t)di * d && y.wv == y.wk + (size_t)di * d) {
+            CSD_TRY(wide_linear(M, y.wq, nullptr, 3 * di, d, m, M->wxs_x, M->wssq, cnt, M->wqkv, 3 * di, EPI_STORE, nullptr, 0,
+                                nullptr, nullptr, st));
+        } else {
+            const __nv_bfloat16* w3[3] = {y.wq, y.wk, y.wv};
+            for (int i = 0; i < 3; ++i)
+                CSD_TRY(wide_linear(M, w3[i], nullptr, di, d, m, M->wxs_x, M->wssq, cnt, M->wqkv + (size_t)i * di, 3 * di,
+                                    EPI_STORE, nullptr, 0, nullptr, nullptr, st));
+        }
+        {   // rotate q and k, append k and v of all rows; the sub-blocks below then only read the cache
+            ProfScope ps(M, 2, st);
+            rope_append_kernel<<<dim3(m, H), 64, 0, st>>>(M->wqkv, 3 * di, c.arch == 0 ? 0 : -1, di, 2 * di, Dh, kv_len, c.max_seq,
+                                                          c.arch == 0 ? M->rope_c : nullptr, c.arch == 0 ? M->rope_s : nullptr, Kl, Vl);
+            count_launch();
+        }
+        if (l + 1 == c.n_layers) break;    // the cache is complete; the rest of the last layer feeds nothing
+        CSD_TRY(wide_attention(M, M->wqkv, 3 * di, m, Kl, Vl, c.max_seq, kv_len + 1, true,
+                               c.arch == 1 ? M->dec_bias : nullptr, c.max_seq, c.max_seq - 1, kv_len, M->wattn, st));
+        CSD_TRY(launch_wide_split(M->wattn, di, di, m, nullptr, M->wxs_attn, nullptr, st));
+        const __nv_bfloat16* after_o = c.arch == 1 ? y.norm_x : y.norm2;
+        CSD_TRY(wide_linear(M, y.wo, nullptr, d, di, m, M->wxs_attn, nullptr, 0, M->wx, d, EPI_ADD, M->wxs_x, d, after_o,
+                            M->wssq, st));
+        cnt = wide_ssq_pieces(m, d, di, false);
+        if (c.arch == 1) {
+            CSD_TRY(wide_linear(M, y.xq, nullptr, di, d, m, M->wxs_x, M->wssq, cnt, M->wqkv, 3 * di, EPI_STORE, nullptr, 0,
+                                nullptr, nullptr, st));
+            CSD_TRY(wide_attention(M, M->wqkv, 3 * di, m, M->xk + (size_t)l * M->layer_x, M->xv + (size_t)l * M->layer_x,
+                                   c.max_enc_len, M->enc_len, false, nullptr, 0, 0, 0, M->wattn, st));
+            CSD_TRY(launch_wide_split(M->wattn, di, di, m, nullptr, M->wxs_attn, nullptr, st));
+            CSD_TRY(wide_linear(M, y.xo, nullptr, d, di, m, M->wxs_attn, nullptr, 0, M->wx, d, EPI_ADD, M->wxs_x, d, y.norm2,
+                                M->wssq, st));
+            cnt = wide_ssq_pieces(m, d, di, false);
+        }
+        CSD_TRY(wide_linear(M, y.wgate, y.wup, ff, d, m, M->wxs_x, M->wssq, cnt, M->wact, ff,
+                            c.arch == 0 ? EPI_SWIGLU : EPI_GEGLU, M->wxs_act, ff, nullptr, nullptr, st));
+        CSD_TRY(wide_linear(M, y.wdown, nullptr, d, ff, m, M->wxs_act, nullptr, 0, M->wx, d, EPI_ADD, M->wxs_x, d,
+                            M->dec[l + 1].norm1, M->wssq, st));
+        cnt = wide_ssq_pieces(m, d, ff, false);
+    }
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
+}
+
 }  // namespace csd
 
 using namespace csd;
@@ -340,6 +455,13 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
     M->xs_x = (__nv_bfloat16*)(ws + L.xs_x); M->xs_attn = (__nv_bfloat16*)(ws + L.xs_attn);
     M->xs_act = (__nv_bfloat16*)(ws + L.xs_act); M->ssq_x = (float*)(ws + L.ssq_x);
     M->status = status;
+    M->wide = L.wide;
+    if (L.wide) {
+        M->wx = (float*)(ws + L.wx); M->wqkv = (float*)(ws + L.wqkv); M->wattn = (float*)(ws + L.wattn);
+        M->wact = (float*)(ws + L.wact); M->wxs_x = (__nv_bfloat16*)(ws + L.wxs_x);
+        M->wxs_attn = (__nv_bfloat16*)(ws + L.wxs_attn); M->wxs_act = (__nv_bfloat16*)(ws + L.wxs_act);
+        M->wssq = (float*)(ws + L.wssq);
+    }
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.xs_tmp - L.gemm_tickets, st);
     if (e != cudaSuccess) { delete M; return note_cuda(e); }
@@ -457,6 +579,28 @@ extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_token
     }
     CSD_CUDA(cudaGetLastError());
     M->enc_len = n;
+    return CSD_OK;
+}
+
+extern "C" csd_status csd_prefill(csd_model* M, const int32_t* tokens_dev, int n, int kv_len, void* stream) {
+    if (!M || !tokens_dev || n < 1 || kv_len < 0) return CSD_ERR_INVALID_ARG;
+    const csd_model_config& c = M->cfg;
+    if (kv_len + n > c.max_seq) return CSD_ERR_CAPACITY;
+    if (c.arch == 1 && M->enc_len < 1) return CSD_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    const int small = c.max_rows < CSD_MAX_ROWS ? c.max_rows : CSD_MAX_ROWS;
+    for (int from = 0; from < n;) {
+        int cnt = n - from;
+        // wide passes while more than one review block is left, review-sized blocks otherwise
+        if (M->wide && gemm_path() != 1 && cnt > small) {
+            if (cnt > CSD_WIDE_ROWS) cnt = CSD_WIDE_ROWS;
+            CSD_TRY(wide_decoder_pass(M, tokens_dev + from, cnt, kv_len + from, st));
+        } else {
+            if (cnt > small) cnt = small;
+            CSD_TRY(csd_review_forward(M, tokens_dev + from, cnt, kv_len + from, nullptr, stream));
+        }
+        from += cnt;
+    }
     return CSD_OK;
 }
 

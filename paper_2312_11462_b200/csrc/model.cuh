@@ -35,6 +35,11 @@ struct csd_model {
     float* ssq_x = nullptr;             // [ssq_x_cnt][rows] pieces of the sums of squares of the residual rows
     int ssq_x_cnt = 0;                  // pieces the GEMM that last produced the residual rows wrote
     int* status = nullptr;
+    // wide blocks (prompt prefill, encoder pass): up to CSD_WIDE_ROWS rows per pass over the weights
+    bool wide = false;                  // every layer matrix takes the wide-block kernel
+    float *wx = nullptr, *wqkv = nullptr, *wattn = nullptr, *wact = nullptr;            // [128][d], [128][3 d_inner], ...
+    __nv_bfloat16 *wxs_x = nullptr, *wxs_attn = nullptr, *wxs_act = nullptr;            // two-term rows [2][128][K]
+    float* wssq = nullptr;              // pieces of the rows' sums of squares
     // optional per-kernel-class timing (csd_model_profile): event pairs around every launch
     bool prof = false;
     std::vector<cudaEvent_t> prof_ev;      // start, stop, start, stop, ...

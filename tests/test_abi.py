@@ -67,7 +67,9 @@ def test_argument_checks_return_before_any_launch(b):
     assert L.csd_spec_accept(256, None, None, 256, 1, 1, 8, 1.0, 1.0, 0, 0, 256, 256, 256, 16, None) == 3
     assert L.csd_spec_accept(256, None, None, 256, 0, 1, 8, 1.0, 1.0, 0, 0, 256, 256, 256, 16, None) == 0  # no rows
     assert L.csd_linear(256, 8, 12, 256, 1, 256, 256, 1 << 20, None) == 1      # K not a multiple of 8
-    assert L.csd_linear(256, 8, 16, 256, 18, 256, 256, 1 << 20, None) == 1     # too many rows
+    assert L.csd_linear(256, 8, 16, 256, 129, 256, 256, 1 << 20, None) == 1    # too many rows
+    assert L.csd_linear(256, 8, 16, 256, 18, 256, 256, 1 << 20, None) == 8     # a wide block needs a large matrix
+    assert L.csd_prefill(None, 256, 4, 0, None) == 1
     assert L.csd_mag_draft(None, 256, 1, 1, 256, None) == 1
     assert L.csd_spec_accept_workspace_bytes(64, 16, 128256) > 0
     assert L.csd_cascade_workspace_bytes(32000, 4, 448, 128, 16) > 0

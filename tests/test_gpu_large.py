@@ -236,3 +236,45 @@ def test_t5xxl_width_sampled_horizontal_cascade(b, orc):
             first = int(np.nonzero(got != want)[0][0])
             assert ost["near_ties"] > 0 and ost["first_near_tie"] <= first, (seed, first, ost)
     assert exact >= 1
+
+
+def test_wide_prefill_leaves_the_cache_a_review_needs(b, orc):
+    """csd_prefill at the 7B width (wide blocks of up to 128 rows, two-term activations): the review
+    block that follows must meet the stated tolerance against the oracle, which forwards every
+    token the plain way; so must a second block after a second prefill that starts mid-cache, and
+    the result must not depend on how the prompt was cut into prefill calls beyond that tolerance."""
+    shape = llama_shape(3, 4096, 32, 11008, 32000, 320)
+    blob = workloads.make_weights(shape, seed=100, device="cuda")
+    seq = workloads.make_prompt(shape.vocab, 300, seed=1000)
+    # the oracle takes the prompt in blocks of its own choice (block partition does not change its result)
+    om2 = orc.Model(shape, orc.blob_to_u16(blob))
+    refs = {}
+    pos = 0
+    for cut in (150, 155, 290, 295):
+        while pos < cut:
+            n = min(17, cut - pos)
+            out = om2.review_forward(seq[pos:pos + n], pos)
+            pos += n
+        refs[cut] = out
+    gm = b.Model(shape, blob)
+    dev = to_dev_i32(seq)
+    gm.csd_prefill(dev[:150].contiguous(), 0)                        # 128 wide + 22 (17 + 5 review-sized)
+    g = gm.csd_review_forward(dev[150:155].contiguous(), 150).cpu().numpy()
+    assert rel_l2(g, refs[155]) <= LOGIT_REL_L2, rel_l2(g, refs[155])
+    assert np.abs(g - refs[155]).max() <= LOGIT_MAX_ABS
+    gm.csd_prefill(dev[155:290].contiguous(), 155)                   # starts mid-cache: 128 wide + 7
+    g = gm.csd_review_forward(dev[290:295].contiguous(), 290).cpu().numpy()
+    assert rel_l2(g, refs[295]) <= LOGIT_REL_L2, rel_l2(g, refs[295])
+    # the same prompt through the review kernels only
+    gm2 = b.Model(shape, blob)
+    p = 0
+    while p < 150:
+        n = min(17, 150 - p)
+        gm2.csd_review_forward(dev[p:p + n].contiguous(), p, append_only=True)
+        p += n
+    g2 = gm2.csd_review_forward(dev[150:155].contiguous(), 150).cpu().numpy()
+    g1 = b.Model(shape, blob)
+    g1.csd_prefill(dev[:150].contiguous(), 0)
+    g1o = g1.csd_review_forward(dev[150:155].contiguous(), 150).cpu().numpy()
+    assert rel_l2(g1o, g2) <= LOGIT_REL_L2
+    assert b.csd_device_status() == 0

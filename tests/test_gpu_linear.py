@@ -54,3 +54,26 @@ def test_head_shape_and_uneven_ranges(b, orc):
     # that leave ranges of unequal length, a K tail and fewer K blocks than a stage holds
     for m, N, K in ((5, 32000, 4096), (3, 20011, 1032), (8, 2371, 4104), (2, 2368, 72)):
         case(b, orc, m, N, K, seed=N + m)
+
+
+def test_wide_blocks(orc):
+    # 18 to 128 rows: the wide-block tensor-core kernel of the prefill.  Each fp32 value enters as two
+    # bf16 terms (16 mantissa bits), so the bound is 2^-17-sized, not the 5e-6 of the review kernels.
+    require_gpu()
+    from paper_2312_11462_b200 import binding as b
+    for m, N, K in ((18, 4096, 4096), (64, 12288, 4096), (128, 4096, 11008), (127, 32000, 4096), (33, 4099, 520),
+                    (100, 20011, 1032), (128, 2371, 4104)):
+        g = torch.Generator(device="cuda")
+        g.manual_seed(m + N)
+        W = (0.05 * torch.randn(N, K, generator=g, device="cuda")).to(torch.bfloat16)
+        X = torch.randn(m, K, generator=g, device="cuda")
+        Y = b.csd_linear(W, X)
+        assert torch.equal(Y, b.csd_linear(W, X))
+        rows = [0, 1, m // 2, m - 2, m - 1]                 # the oracle on a few rows bounds its cost
+        ref = orc.linear(orc.blob_to_u16(W).reshape(N, K), X[rows].cpu().numpy())
+        got = Y[rows].cpu().numpy()
+        assert rel_l2(got, ref) < 3e-5, (m, N, K, rel_l2(got, ref))
+        # every row against a float64 product on the GPU side of the harness (torch matmul as the library step)
+        full = (X.double() @ W.double().T)
+        assert float((Y.double() - full).norm() / full.norm()) < 3e-5
+    assert b.csd_device_status() == 0
