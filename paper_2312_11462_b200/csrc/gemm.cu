@@ -402,7 +402,12 @@ static LinearWs linear_ws(int m, int N, int K) {
     size_t off = 0;
     const int rows = m > CSD_MAX_ROWS ? CSD_WIDE_ROWS : CSD_MAX_ROWS;
     w.tickets = off; off += align_up((size_t)linear_ticket_count(N) * sizeof(unsigned), 256);
-    w.partial = off; off += linear_scratch_bytes(m > CSD_MAX_ROWS ? CSD_MAX_ROWS : m, N, K, false);
+    w.partial = off;
+    {
+        size_t pb = linear_scratch_bytes(m > CSD_MAX_ROWS ? CSD_MAX_ROWS : m, N, K, false);
+        if (m > CSD_MAX_ROWS && wide_partial_bytes(m, N, K, false) > pb) pb = wide_partial_bytes(m, N, K, false);
+        off += pb;
+    }
     w.xs = off;      off += align_up((size_t)3 * rows * K * 2, 256);
     w.ssq = off;     off += align_up((size_t)split_ssq_entries(K) * rows * sizeof(float), 256);
     w.total = off;
@@ -430,7 +435,7 @@ extern "C" csd_status csd_linear(const void* W_bf16_dev, int N, int K, const flo
         if (s != CSD_OK) return s;
         WideArgs wa;
         wa.W = (const __nv_bfloat16*)W_bf16_dev; wa.N = N; wa.K = K; wa.m = m; wa.xs = (const __nv_bfloat16*)(ws + w.xs);
-        wa.Y = Y_dev; wa.ldy = N; wa.epilogue = EPI_STORE;
+        wa.Y = Y_dev; wa.ldy = N; wa.epilogue = EPI_STORE; wa.partial = (float*)(ws + w.partial);
         return launch_linear_wide(wa, (cudaStream_t)stream);
     }
     LinearArgs a;

@@ -33,10 +33,12 @@ struct WideArgs {
     int out_ld = 0;
     const __nv_bfloat16* out_gain = nullptr;
     float* out_ssq = nullptr;            // optional: [wide_ssq_pieces(...)][m] pieces of the sums of squares of the rows of Y
+    float* partial = nullptr;            // scratch of wide_partial_bytes(...) for K-partitioned launches (optional)
 };
 bool wide_supported(int m, int N, int K, bool dual);
 int wide_ssq_pieces(int m, int N, int K, bool dual);
 int wide_ssq_capacity(int N);
+size_t wide_partial_bytes(int m, int N, int K, bool dual);
 int wide_split_pieces(int K);
 csd_status launch_wide_split(const float* X, int ldx, int K, int m, const __nv_bfloat16* gain, __nv_bfloat16* xs,
                              float* ssq, cudaStream_t st);

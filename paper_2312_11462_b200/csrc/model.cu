@@ -137,7 +137,7 @@ static size_t walk_blob(const csd_model_config& c, const __nv_bfloat16* base, cs
 struct WsLayout {
     size_t kcache, vcache, xk, xv, ek, ev, x, qkv, attn, act, xenc, qkv_enc, rope_c, rope_s, dec_bias, enc_bias,
         buckets, gemm_partial, gemm_tickets, xs_tmp, ssq_tmp, xs_x, xs_attn, xs_act, ssq_x,
-        wx, wqkv, wattn, wact, wxs_x, wxs_attn, wxs_act, wssq, total;
+        wx, wqkv, wattn, wact, wxs_x, wxs_attn, wxs_act, wssq, wpart, total;
     bool wide;
     size_t layer_kv, layer_x;
 };
@@ -187,6 +187,9 @@ static WsLayout ws_layout(const csd_model_config& c) {
         size_t pieces = (size_t)wide_ssq_capacity((int)d);
         if ((size_t)wide_split_pieces((int)kmax_w) > pieces) pieces = (size_t)wide_split_pieces((int)kmax_w);
         L.wssq = put(pieces * WR * 4);
+        size_t pb = wide_partial_bytes((int)WR, (int)d, (int)di, false);
+        if (wide_partial_bytes((int)WR, (int)d, (int)ff, false) > pb) pb = wide_partial_bytes((int)WR, (int)d, (int)ff, false);
+        L.wpart = put(pb > 0 ? pb : 256);
     }
     if (c.arch == 0) {
         L.rope_c = put((size_t)c.max_seq * (Dh / 2) * 4);
@@ -309,6 +312,7 @@ static csd_status wide_linear(csd_model* M, const __nv_bfloat16* W, const __nv_b
     WideArgs a;
     a.W = W; a.W2 = W2; a.N = N; a.K = K; a.m = m; a.xs = xs; a.ssq = ssq; a.ssq_cnt = ssq_cnt; a.eps = M->cfg.norm_eps;
     a.Y = Y; a.ldy = ldy; a.epilogue = epi; a.out_xs = out_xs; a.out_ld = out_ld; a.out_gain = out_gain; a.out_ssq = out_ssq;
+    a.partial = M->wpart;
     ProfScope ps(M, 0, st);
     if (M->prof) M->prof_gemm_bytes += (double)N * K * 2.0 * (W2 ? 2.0 : 1.0);
     return launch_linear_wide(a, st);
@@ -460,7 +464,7 @@ extern "C" csd_status csd_model_create(const csd_model_config* cfg, const void* 
         M->wx = (float*)(ws + L.wx); M->wqkv = (float*)(ws + L.wqkv); M->wattn = (float*)(ws + L.wattn);
         M->wact = (float*)(ws + L.wact); M->wxs_x = (__nv_bfloat16*)(ws + L.wxs_x);
         M->wxs_attn = (__nv_bfloat16*)(ws + L.wxs_attn); M->wxs_act = (__nv_bfloat16*)(ws + L.wxs_act);
-        M->wssq = (float*)(ws + L.wssq);
+        M->wssq = (float*)(ws + L.wssq); M->wpart = (float*)(ws + L.wpart);
     }
     cudaStream_t st = (cudaStream_t)stream;
     cudaError_t e = cudaMemsetAsync(ws + L.gemm_tickets, 0, L.xs_tmp - L.gemm_tickets, st);

@@ -40,6 +40,7 @@ struct csd_model {
     float *wx = nullptr, *wqkv = nullptr, *wattn = nullptr, *wact = nullptr;            // [128][d], [128][3 d_inner], ...
     __nv_bfloat16 *wxs_x = nullptr, *wxs_attn = nullptr, *wxs_act = nullptr;            // two-term rows [2][128][K]
     float* wssq = nullptr;              // pieces of the rows' sums of squares
+    float* wpart = nullptr;             // partial planes of K-partitioned wide GEMMs
     // optional per-kernel-class timing (csd_model_profile): event pairs around every launch
     bool prof = false;
     std::vector<cudaEvent_t> prof_ev;      // start, stop, start, stop, ...
