@@ -399,6 +399,66 @@ static csd_status wide_decoder_pass(csd_model* M, const int32_t* tokens, int m, 
     return CSD_OK;
 }
 
+// Encoder pass (arch 1) in wide blocks: every layer projects q|k|v of all rows, appends K/V, then
+// runs attention, output projection and feed-forward block by block; afterwards the cross-attention
+// K/V of every decoder layer.
+static csd_status wide_encoder(csd_model* M, int n, cudaStream_t st) {
+    const csd_model_config& c = M->cfg;
+    const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, ff = c.d_ff, E = c.max_enc_len, WR = CSD_WIDE_ROWS;
+    for (int l = 0; l < c.n_enc_layers; ++l) {
+        const LayerW& y = M->enc[l];
+        const bool fused = y.wk == y.wq + (size_t)di * d && y.wv == y.wk + (size_t)di * d;
+        for (int r0 = 0; r0 < n; r0 += WR) {
+            const int m = n - r0 < WR ? n - r0 : WR;
+            CSD_TRY(launch_wide_split(M->xenc + (size_t)r0 * d, d, d, m, y.norm1, M->wxs_x, M->wssq, st));
+            const int cnt = wide_split_pieces(d);
+            float* out = M->qkv_enc + (size_t)r0 * 3 * di;
+            if (fused) {
+                CSD_TRY(wide_linear(M, y.wq, nullptr, 3 * di, d, m, M->wxs_x, M->wssq, cnt, out, 3 * di, EPI_STORE, nullptr, 0,
+                                    nullptr, nullptr, st));
+            } else {
+                const __nv_bfloat16* w3[3] = {y.wq, y.wk, y.wv};
+                for (int i = 0; i < 3; ++i)
+                    CSD_TRY(wide_linear(M, w3[i], nullptr, di, d, m, M->wxs_x, M->wssq, cnt, out + (size_t)i * di, 3 * di,
+                                        EPI_STORE, nullptr, 0, nullptr, nullptr, st));
+            }
+        }
+        rope_append_kernel<<<dim3(n, H), 64, 0, st>>>(M->qkv_enc, 3 * di, -1, di, 2 * di, Dh, 0, E, nullptr, nullptr, M->ek, M->ev);
+        count_launch();
+        for (int r0 = 0; r0 < n; r0 += WR) {
+            const int m = n - r0 < WR ? n - r0 : WR;
+            float* xr = M->xenc + (size_t)r0 * d;
+            CSD_TRY(wide_attention(M, M->qkv_enc + (size_t)r0 * 3 * di, 3 * di, m, M->ek, M->ev, E, n, false, M->enc_bias,
+                                   2 * E - 1, E - 1, r0, M->wattn, st));
+            CSD_TRY(launch_wide_split(M->wattn, di, di, m, nullptr, M->wxs_attn, nullptr, st));
+            CSD_TRY(wide_linear(M, y.wo, nullptr, d, di, m, M->wxs_attn, nullptr, 0, xr, d, EPI_ADD, M->wxs_x, d, y.norm2,
+                                M->wssq, st));
+            CSD_TRY(wide_linear(M, y.wgate, y.wup, ff, d, m, M->wxs_x, M->wssq, wide_ssq_pieces(m, d, di, false), M->wact, ff,
+                                EPI_GEGLU, M->wxs_act, ff, nullptr, nullptr, st));
+            CSD_TRY(wide_linear(M, y.wdown, nullptr, d, ff, m, M->wxs_act, nullptr, 0, xr, d, EPI_ADD, nullptr, 0, nullptr,
+                                nullptr, st));
+        }
+    }
+    for (int l = 0; l < c.n_layers; ++l) {
+        const LayerW& y = M->dec[l];
+        for (int r0 = 0; r0 < n; r0 += WR) {
+            const int m = n - r0 < WR ? n - r0 : WR;
+            CSD_TRY(launch_wide_split(M->xenc + (size_t)r0 * d, d, d, m, M->enc_final_norm, M->wxs_x, M->wssq, st));
+            const int cnt = wide_split_pieces(d);
+            float* out = M->qkv_enc + (size_t)r0 * 3 * di;
+            CSD_TRY(wide_linear(M, y.xk, nullptr, di, d, m, M->wxs_x, M->wssq, cnt, out + di, 3 * di, EPI_STORE, nullptr, 0, nullptr,
+                                nullptr, st));
+            CSD_TRY(wide_linear(M, y.xv, nullptr, di, d, m, M->wxs_x, M->wssq, cnt, out + 2 * di, 3 * di, EPI_STORE, nullptr, 0,
+                                nullptr, nullptr, st));
+        }
+        rope_append_kernel<<<dim3(n, H), 64, 0, st>>>(M->qkv_enc, 3 * di, -1, di, 2 * di, Dh, 0, E, nullptr, nullptr,
+                                                      M->xk + (size_t)l * M->layer_x, M->xv + (size_t)l * M->layer_x);
+        count_launch();
+    }
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
+}
+
 }  // namespace csd
 
 using namespace csd;
@@ -546,6 +606,11 @@ extern "C" csd_status csd_encoder_forward(csd_model* M, const int32_t* enc_token
     const int CH = 16;
     embed_kernel<<<n, 128, 0, st>>>(enc_tokens_dev, M->embed, c.vocab, d, M->xenc, M->status);
     count_launch();
+    if (M->wide && gemm_path() != 1 && n > CSD_MAX_ROWS) {      // large model: wide blocks
+        CSD_TRY(wide_encoder(M, n, st));
+        M->enc_len = n;
+        return CSD_OK;
+    }
     for (int l = 0; l < c.n_enc_layers; ++l) {
         const LayerW& y = M->enc[l];
         for (int r0 = 0; r0 < n; r0 += CH) {
