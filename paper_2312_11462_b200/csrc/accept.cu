@@ -16,6 +16,7 @@
 //            reciprocal formed once.
 #include "common.cuh"
 #include "philox.cuh"
+#include <math.h>
 #include <mutex>
 
 namespace csd {
@@ -251,40 +252,64 @@ __device__ __forceinline__ double block_sum_ordered(double v, double* s_warp) {
     return tot;
 }
 
-// exp(x) for x <= 0 in fp64: x = n ln2 + r with |r| <= ln2 / 2, e^r by its Taylor series to r^11
-// (remainder below 2.3e-13 relative), times 2^n through the exponent field.  Below -708 the
-// result is 0 (the true value is under the smallest normal number).
-__device__ __forceinline__ double exp_neg(double x) {
+// exp(x) for x <= 0 in fp64 by table and polynomial: x = (64 m + j) ln2/64 + r with |r| <= ln2/128,
+// exp(x) = 2^m * 2^(j/64) * e^r; the 64 table entries are correctly rounded doubles made on the host,
+// e^r is its Taylor series to r^5 (remainder below 4e-17), 2^m goes through the exponent field.
+// Relative error about 3e-16.  Below -708 the result is 0 (under the smallest normal number).
+__constant__ double c_exp2_table[64];
+__device__ __forceinline__ void exp_table_to_shared(double* s_tab) {
+    for (int i = threadIdx.x; i < 64; i += blockDim.x) s_tab[i] = c_exp2_table[i];
+    __syncthreads();
+}
+__device__ __forceinline__ double exp_neg(double x, const double* __restrict__ s_tab) {
     if (!(x > -708.0)) return 0.0;
-    const double n = rint(x * 1.4426950408889634);
-    double r = fma(-n, 6.93147180369123816490e-01, x);        // ln 2, high part (low bits clear)
-    r = fma(-n, 1.90821492927058770002e-10, r);               // ln 2, low part
-    double p = 1.0 / 39916800.0;
-    p = fma(p, r, 1.0 / 3628800.0);
-    p = fma(p, r, 1.0 / 362880.0);
-    p = fma(p, r, 1.0 / 40320.0);
-    p = fma(p, r, 1.0 / 5040.0);
-    p = fma(p, r, 1.0 / 720.0);
-    p = fma(p, r, 1.0 / 120.0);
+    const double nf = rint(x * 92.33248261689366);           // 64 / ln 2
+    double r = fma(-nf, 0.01083042468962958, x);              // ln 2 / 64, high part (low 22 bits clear: nf * high is exact)
+    r = fma(-nf, 6.619564634077006e-12, r);                   // ln 2 / 64, low part
+    const int n = (int)nf;
+    double p = 1.0 / 120.0;
     p = fma(p, r, 1.0 / 24.0);
     p = fma(p, r, 1.0 / 6.0);
     p = fma(p, r, 0.5);
     p = fma(p, r, 1.0);
-    p = fma(p, r, 1.0);
-    const long long bits = __double_as_longlong(p) + ((long long)n << 52);   // n >= -1022: stays a normal number
+    p *= r;                                                   // e^r - 1
+    const double tj = s_tab[n & 63];
+    const double v = fma(tj, p, tj);
+    const long long bits = __double_as_longlong(v) + ((long long)(n >> 6) << 52);   // m >= -1022: stays a normal number
     return __longlong_as_double(bits);
 }
 
+// eight consecutive logits of a vector (two 16-byte loads when the vector allows it); past V: -inf
+__device__ __forceinline__ void load8(const float* __restrict__ src, int e0, int V, bool vec, float (&v)[8]) {
+    if (vec && e0 + 7 < V) {
+        const float4 a = __ldcs(reinterpret_cast<const float4*>(src + e0));
+        const float4 b = __ldcs(reinterpret_cast<const float4*>(src + e0 + 4));
+        v[0] = a.x; v[1] = a.y; v[2] = a.z; v[3] = a.w; v[4] = b.x; v[5] = b.y; v[6] = b.z; v[7] = b.w;
+    } else {
+#pragma unroll
+        for (int j = 0; j < 8; ++j) v[j] = e0 + j < V ? __ldcs(src + e0 + j) : -INFINITY;
+    }
+}
+
 struct ResidualCtx {
-    const float* t; const float* d;
+    const float* t; const float* d; const double* tab;
     double max_t, max_q, invT, inv_zt, inv_zq;
     int mode, x;
 };
 __device__ __forceinline__ double residual_at(const ResidualCtx& c, int e) {
-    const double p = exp_neg(((double)c.t[e] - c.max_t) * c.invT) * c.inv_zt;
+    const double p = exp_neg(((double)c.t[e] - c.max_t) * c.invT, c.tab) * c.inv_zt;
     if (c.mode == MODE_TARGET_ONLY) return p;
     const double q = c.mode == MODE_RESID_POINT ? (e == c.x ? 1.0 : 0.0)
-                                                : exp_neg(((double)c.d[e] - c.max_q) * c.invT) * c.inv_zq;
+                                                : exp_neg(((double)c.d[e] - c.max_q) * c.invT, c.tab) * c.inv_zq;
+    const double r = p - q;
+    return r > 0.0 ? r : 0.0;
+}
+
+__device__ __forceinline__ double residual_of(const ResidualCtx& c, int e, float tv, float dv) {
+    const double p = exp_neg(((double)tv - c.max_t) * c.invT, c.tab) * c.inv_zt;
+    if (c.mode == MODE_TARGET_ONLY) return p;
+    const double q = c.mode == MODE_RESID_POINT ? (e == c.x ? 1.0 : 0.0)
+                                                : exp_neg(((double)dv - c.max_q) * c.invT, c.tab) * c.inv_zq;
     const double r = p - q;
     return r > 0.0 ? r : 0.0;
 }
@@ -298,17 +323,23 @@ resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, in
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
+    __shared__ double s_tab[64];
+    exp_table_to_shared(s_tab);
     const double invT = 1.0 / (double)temperature;
     const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
     const float* d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
     const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
     double sp = 0.0, sq = 0.0;
+    {
+        static_assert(RS_PER_THREAD == 8, "load8 covers a thread's entries");
+        const bool vec = (V % 4 == 0) && ((((uintptr_t)t) & 15) == 0) && (!d || (((uintptr_t)d) & 15) == 0);
+        float tv[8], dv[8];
+        load8(t, e0, V, vec, tv);
+        if (d) load8(d, e0, V, vec, dv);
 #pragma unroll
-    for (int j = 0; j < RS_PER_THREAD; ++j) {
-        const int e = e0 + j;
-        if (e < V) {
-            sp += exp_neg(((double)t[e] - ri.max_t) * invT);
-            if (d) sq += exp_neg(((double)d[e] - ri.max_q) * invT);
+        for (int j = 0; j < RS_PER_THREAD; ++j) {
+            sp += exp_neg(((double)tv[j] - ri.max_t) * invT, s_tab);      // -inf (past V) gives 0
+            if (d) sq += exp_neg(((double)dv[j] - ri.max_q) * invT, s_tab);
         }
     }
     sp = block_sum_ordered(sp, s_warp);
@@ -351,6 +382,8 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     __shared__ double s_d[2];    // target, base
     __shared__ int s_i[3];       // chunk, mode, forced-last flag
     __shared__ int s_pick, s_last, s_is_last;
+    __shared__ double s_tab[64];
+    exp_table_to_shared(s_tab);
     const double2* zrow = zpart + (long long)row * nchunk;
     double* rrow = rpart + (long long)row * nchunk;
     const double Zp = zsum[row].x, Zq = zsum[row].y;
@@ -359,13 +392,17 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     c.d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
     c.max_t = ri.max_t; c.max_q = ri.max_q; c.invT = 1.0 / (double)temperature;
     c.inv_zt = 1.0 / Zp; c.inv_zq = Zq > 0.0 ? 1.0 / Zq : 0.0;
-    c.mode = ri.mode; c.x = ri.x;
+    c.mode = ri.mode; c.x = ri.x; c.tab = s_tab;
     {
         const int e0 = chunk * RS_CHUNK + threadIdx.x * RS_PER_THREAD;
+        const bool vec = (V % 4 == 0) && ((((uintptr_t)c.t) & 15) == 0) && (!c.d || (((uintptr_t)c.d) & 15) == 0);
+        float tv[8], dv[8];
+        load8(c.t, e0, V, vec, tv);
+        if (c.d) load8(c.d, e0, V, vec, dv);
         double sr = 0.0;
 #pragma unroll
         for (int j = 0; j < RS_PER_THREAD; ++j)
-            if (e0 + j < V) sr += residual_at(c, e0 + j);
+            if (e0 + j < V) sr += residual_of(c, e0 + j, tv[j], c.d ? dv[j] : 0.f);
         sr = block_sum_ordered(sr, s_warp);
         if (threadIdx.x == 0) {
             rrow[chunk] = sr;
@@ -469,6 +506,170 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
     if (threadIdx.x == 0) out_tok[row] = s_pick != 0x7fffffff ? s_pick : (s_last >= 0 ? s_last : 0);
 }
 
+// ---------------------------------------------------------------------------------------------
+// resample, one kernel: a row is a thread-block cluster of up to RF_MAXC CTAs; a CTA keeps its
+// slice of the two logit vectors (position n only) in registers, so global memory is read once.
+// Round 1: per-CTA sums of the exponentials, exchanged through distributed shared memory -> the
+// normalisers.  Round 2: per-CTA residual mass -> total mass S and the CTA whose slice holds
+// u2 * S.  That CTA scans its threads' sums in thread order and picks the entry.  All sums have a
+// fixed order (lanes by xor-shuffle or prefix scan, warps and CTAs in index order).
+// ---------------------------------------------------------------------------------------------
+constexpr int RF_THREADS = 512, RF_PER = 16, RF_SLICE = RF_THREADS * RF_PER, RF_MAXC = 16;
+constexpr int RF_USE_MAXC = 8;   // larger clusters run (one per GPC at a time) but lose to the two-pass kernels: 199 us against 145 at V = 128256
+
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync_all() {
+    asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ double cluster_read_f64(const double* local, uint32_t rank) {
+    uint32_t a = (uint32_t)__cvta_generic_to_shared(local), r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(a), "r"(rank));
+    double v;
+    asm volatile("ld.shared::cluster.f64 %0, [%1];" : "=d"(v) : "r"(r) : "memory");
+    return v;
+}
+
+// ordered sum over the CTA; the result is valid in every thread
+__device__ __forceinline__ double rf_block_sum(double v, double* s_warp) {
+    v = warp_sum(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    __syncthreads();
+    if (lane == 0) s_warp[warp] = v;
+    __syncthreads();
+    double tot = 0.0;
+    for (int w = 0; w < RF_THREADS / 32; ++w) tot += s_warp[w];
+    return tot;
+}
+
+__global__ void __launch_bounds__(RF_THREADS, 1)
+resample_fused_kernel(const float* __restrict__ tl, const float* __restrict__ dl, int k, int V, float temperature,
+                      const RowInfo* __restrict__ info, int csize, int* __restrict__ out_tok) {
+    const int row = blockIdx.x / csize;
+    const uint32_t rank = cluster_rank();
+    const RowInfo ri = info[row];
+    if (ri.mode == MODE_DONE) return;                 // (the same decision in every CTA of the cluster)
+    __shared__ double s_warp[RF_THREADS / 32];
+    __shared__ double s_ex[2];                        // this CTA's contribution to the current exchange
+    __shared__ double s_scan[RF_THREADS / 32];
+    __shared__ int s_pick, s_last;
+    __shared__ double s_tab[64];
+    exp_table_to_shared(s_tab);
+    const double invT = 1.0 / (double)temperature;
+    const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
+    const float* d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
+    const int e0 = (int)rank * RF_SLICE + threadIdx.x * RF_PER;
+    // ---- this thread's entries, read once; their exponentials stay in registers for both rounds
+    double et[RF_PER], ed[RF_PER];
+    const bool vec = (V % 4 == 0) && ((((uintptr_t)t) & 15) == 0) && (!d || (((uintptr_t)d) & 15) == 0);
+    double sp = 0.0, sq = 0.0;
+#pragma unroll
+    for (int j = 0; j < RF_PER; j += 4) {
+        const int e = e0 + j;
+        float tv[4], dv[4];
+        if (vec && e + 3 < V) {
+            const float4 a = __ldcs(reinterpret_cast<const float4*>(t + e));
+            tv[0] = a.x; tv[1] = a.y; tv[2] = a.z; tv[3] = a.w;
+            if (d) {
+                const float4 b = __ldcs(reinterpret_cast<const float4*>(d + e));
+                dv[0] = b.x; dv[1] = b.y; dv[2] = b.z; dv[3] = b.w;
+            } else { dv[0] = dv[1] = dv[2] = dv[3] = -INFINITY; }
+        } else {
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                tv[i] = e + i < V ? __ldcs(t + e + i) : -INFINITY;
+                dv[i] = (d && e + i < V) ? __ldcs(d + e + i) : -INFINITY;
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            et[j + i] = exp_neg(((double)tv[i] - ri.max_t) * invT, s_tab);   // -inf (past V) gives 0
+            ed[j + i] = d ? exp_neg(((double)dv[i] - ri.max_q) * invT, s_tab) : 0.0;
+            sp += et[j + i];
+            sq += ed[j + i];
+        }
+    }
+    // ---- round 1: normalisers
+    sp = rf_block_sum(sp, s_warp);
+    sq = rf_block_sum(sq, s_warp);
+    if (threadIdx.x == 0) { s_ex[0] = sp; s_ex[1] = sq; }
+    cluster_sync_all();
+    double Zp = 0.0, Zq = 0.0;
+    for (int c = 0; c < csize; ++c) { Zp += cluster_read_f64(&s_ex[0], (uint32_t)c); Zq += cluster_read_f64(&s_ex[1], (uint32_t)c); }
+    cluster_sync_all();                               // everyone has read before s_ex is reused
+    ResidualCtx cx;
+    cx.t = nullptr; cx.d = nullptr; cx.tab = s_tab; cx.max_t = ri.max_t; cx.max_q = ri.max_q; cx.invT = invT;
+    cx.inv_zt = 1.0 / Zp; cx.inv_zq = Zq > 0.0 ? 1.0 / Zq : 0.0; cx.mode = ri.mode; cx.x = ri.x;
+    auto resid = [&](int j, int mode) -> double {
+        if (e0 + j >= V) return 0.0;
+        const double p = et[j] * cx.inv_zt;
+        if (mode == MODE_TARGET_ONLY) return p;
+        const double q = mode == MODE_RESID_POINT ? (e0 + j == cx.x ? 1.0 : 0.0) : ed[j] * cx.inv_zq;
+        const double r = p - q;
+        return r > 0.0 ? r : 0.0;
+    };
+    // ---- round 2: masses (a second time with the target law itself if the residual is empty)
+    int mode = ri.mode;
+    double local = 0.0, S = 0.0, base = 0.0, my_mass = 0.0;
+    int pick_cta = -1, last_pos = 0;
+    for (int pass = 0; pass < 2; ++pass) {
+        local = 0.0;
+#pragma unroll
+        for (int j = 0; j < RF_PER; ++j) local += resid(j, mode);
+        my_mass = rf_block_sum(local, s_warp);
+        if (threadIdx.x == 0) s_ex[0] = my_mass;
+        cluster_sync_all();
+        S = 0.0;
+        double masses[RF_MAXC];
+        for (int c = 0; c < csize; ++c) { masses[c] = cluster_read_f64(&s_ex[0], (uint32_t)c); S += masses[c]; }
+        cluster_sync_all();
+        const bool empty = !(S > 0.0) || !isfinite(S);
+        if (empty && pass == 0 && mode != MODE_TARGET_ONLY) { mode = MODE_TARGET_ONLY; continue; }
+        const double target = ri.u2 * S;
+        double acc = 0.0;
+        for (int c = 0; c < csize; ++c) {
+            if (masses[c] > 0.0) last_pos = c;
+            if (pick_cta < 0 && acc + masses[c] > target) { pick_cta = c; base = acc; }
+            if (pick_cta < 0) acc += masses[c];
+        }
+        break;
+    }
+    const double target = ri.u2 * S;
+    int forced = 0;
+    if (pick_cta < 0) { pick_cta = last_pos; forced = 1; }
+    if ((int)rank != pick_cta) return;
+    // ---- the picking CTA: exclusive prefix of the threads' sums in thread order, then the entry
+    if (threadIdx.x == 0) { s_pick = 0x7fffffff; s_last = -1; }
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    double incl = local;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const double up = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += up;
+    }
+    if (lane == 31) s_scan[warp] = incl;
+    __syncthreads();
+    double woff = 0.0;
+    for (int w = 0; w < warp; ++w) woff += s_scan[w];
+    double cum = base + woff + (incl - local);
+    int found = 0x7fffffff, my_last = -1;
+#pragma unroll
+    for (int j = 0; j < RF_PER; ++j) {
+        const double r = resid(j, mode);
+        if (r > 0.0) my_last = e0 + j;
+        cum += r;
+        if (!forced && found == 0x7fffffff && r > 0.0 && cum > target) found = e0 + j;
+    }
+    if (found != 0x7fffffff) atomicMin(&s_pick, found);
+    if (my_last >= 0) atomicMax(&s_last, my_last);
+    __syncthreads();
+    if (threadIdx.x == 0) out_tok[row] = s_pick != 0x7fffffff ? s_pick : (s_last >= 0 ? s_last : 0);
+}
+
 struct AcceptLayout {
     size_t part_off, info_off, z_off, zsum_off, r_off, ticket_off, total;
     int nchunk_a, nchunk_r;
@@ -499,6 +700,48 @@ static int accept_sm_count() {
             n = 148;
     }
     return n;
+}
+
+// The table of 2^(j/64), correctly rounded, goes to constant memory once per device.
+static csd_status exp_table_ready() {
+    static bool done[64];
+    static std::mutex mu;
+    int dev = 0;
+    CSD_CUDA(cudaGetDevice(&dev));
+    if (dev < 0 || dev >= 64) return CSD_ERR_UNSUPPORTED;
+    std::lock_guard<std::mutex> lk(mu);
+    if (!done[dev]) {
+        double tab[64];
+        for (int j = 0; j < 64; ++j) tab[j] = exp2((double)j / 64.0);
+        CSD_CUDA(cudaMemcpyToSymbol(c_exp2_table, tab, sizeof(tab)));
+        done[dev] = true;
+    }
+    return CSD_OK;
+}
+
+// Whether clusters of `csize` CTAs of the fused resample kernel can run on this device (sizes above
+// 8 are an opt-in of the hardware); asked once per size.
+static bool fused_resample_ok(int csize) {
+    static int state[RF_MAXC + 1];              // 0 unknown, 1 yes, 2 no
+    if (csize < 1 || csize > RF_USE_MAXC) return false;
+    if (state[csize] == 0) {
+        bool ok = true;
+        if (csize > 8)
+            ok = cudaFuncSetAttribute(resample_fused_kernel, cudaFuncAttributeNonPortableClusterSizeAllowed, 1) == cudaSuccess;
+        if (ok) {
+            cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+            cudaLaunchAttribute attr[1];
+            cfg.gridDim = dim3((unsigned)csize); cfg.blockDim = dim3(RF_THREADS);
+            attr[0].id = cudaLaunchAttributeClusterDimension;
+            attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+            cfg.attrs = attr; cfg.numAttrs = 1;
+            int n = 0;
+            ok = cudaOccupancyMaxActiveClusters(&n, resample_fused_kernel, &cfg) == cudaSuccess && n >= 1;
+        }
+        if (!ok) (void)cudaGetLastError();
+        state[csize] = ok ? 1 : 2;
+    }
+    return state[csize] == 1;
 }
 
 // The three passes on scratch `ws` (accept_layout bytes).  Every word a pass reads is written by an
@@ -541,7 +784,22 @@ static csd_status run_accept(const float* tl, const float* dl_in, const int32_t*
                                     (int*)out_tok, info, tickets, status));
     }
     count_launch(2);
+    const int csize = (V + RF_SLICE - 1) / RF_SLICE;
     if (!greedy) {
+        const csd_status ts = exp_table_ready();
+        if (ts != CSD_OK) return ts;
+    }
+    if (!greedy && fused_resample_ok(csize)) {  // a row fits one cluster: the fused resample kernel
+        cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
+        cudaLaunchAttribute attr[1];
+        cfg.gridDim = dim3((unsigned)(rows * csize)); cfg.blockDim = dim3(RF_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
+        attr[0].id = cudaLaunchAttributeClusterDimension;
+        attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
+        cfg.attrs = attr; cfg.numAttrs = 1;
+        CSD_CUDA(cudaLaunchKernelEx(&cfg, resample_fused_kernel, tl, dl, k, V, temperature, (const RowInfo*)info, csize,
+                                    (int*)out_tok));
+        count_launch();
+    } else if (!greedy) {
         dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
         resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, tickets, L.nchunk_r);
         resample_pick_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, rpart, tickets + rows, L.nchunk_r, out_tok);
