@@ -244,3 +244,53 @@ def cascade_generate(models: Sequence[Model], haystack, bigram_next, K, max_bloc
     if rc:
         raise ValueError(f"orc_cascade_generate failed ({rc})")
     return out[:out_len.value].copy(), margins[:out_len.value].copy(), st.as_dict(n)
+
+
+# --------------------------------------------------------------------------------------------
+# Tree-shaped review (Section 5.1 and Appendix B combine CS Drafting with tree attention: several
+# candidate continuations are reviewed in one pass and the longest accepted path wins).  The plain
+# definition: a node's law is the model's next-token law after the prefix followed by the tokens
+# on the path from the root to that node; greedy acceptance walks down from the root as long as
+# the target's arg-max is among the current node's children.
+# --------------------------------------------------------------------------------------------
+
+def tree_paths(parent: Sequence[int]) -> List[List[int]]:
+    """Row indices from the root (row 0, parent -1) to every node; parents precede children."""
+    paths: List[List[int]] = []
+    for r, p in enumerate(parent):
+        if r == 0:
+            if p != -1:
+                raise ValueError("row 0 is the root (parent -1)")
+            paths.append([0])
+        else:
+            if not (0 <= p < r):
+                raise ValueError("a parent must precede its child")
+            paths.append(paths[p] + [r])
+    return paths
+
+
+def tree_review_forward(model: Model, tokens, parent: Sequence[int], kv_len: int) -> np.ndarray:
+    """Logits [m, vocab]: row r = the model's law after cache[0:kv_len] + the tokens on the path to node r.
+    One plain forward per node (the cache rows from kv_len on are overwritten every time)."""
+    t = _i32(tokens)
+    out = np.zeros((len(t), model.shape.vocab), dtype=np.float32)
+    for r, path in enumerate(tree_paths(parent)):
+        out[r] = model.review_forward(t[path], kv_len)[-1]
+    return out
+
+
+def tree_accept_greedy(logits, tokens, parent: Sequence[int]):
+    """Greedy walk: returns (emitted tokens, rows of the accepted path starting with the root).
+    At the current node the target's arg-max (smallest index on ties) is emitted; if a child holds
+    that token (the child with the smallest row index if several do) the walk moves there."""
+    lg = _f32(logits)
+    t = _i32(tokens)
+    cur, out, path = 0, [], [0]
+    while True:
+        y = int(np.argmax(lg[cur]))
+        out.append(y)
+        nxt = [c for c in range(cur + 1, len(t)) if parent[c] == cur and int(t[c]) == y]
+        if not nxt:
+            return np.asarray(out, dtype=np.int32), path
+        cur = nxt[0]
+        path.append(cur)
