@@ -120,6 +120,28 @@ csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int 
 csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
                               float* logits_out_dev, void* stream);
 
+/* Review of a TREE of drafted tokens in one pass (Section 5.1 and Appendix B combine the method
+ * with tree attention: several candidate continuations hang off a node and the longest accepted
+ * path wins).  Row 0 is the root (the newest token that is not in the cache yet, parent -1); row r
+ * is a child of row parent_host[r] < r.  Row r sits at position kv_len + depth(r), attends to cache
+ * rows [0, kv_len), to its ancestors and to itself, and logits row r is the model's next-token law
+ * after the path from the root to r.  Cache rows [kv_len, kv_len + n_rows) are overwritten with the
+ * rows in index order: only rows of a chain 0, 1, 2, .. (parent[r] = r - 1) leave valid cache entries,
+ * so put the path most likely to be accepted first and re-feed what was accepted elsewhere.
+ * parent_host is read before the call returns.  arch 0 only. */
+csd_status csd_review_forward_tree(csd_model* m, const int32_t* block_tokens_dev, const int32_t* parent_host, int n_rows,
+                                   int kv_len, float* logits_out_dev, void* stream);
+
+/* Greedy acceptance along the tree reviewed by csd_review_forward_tree: starting at the root, the
+ * target's arg-max at the current node is emitted; if a child of the node holds that token (the one
+ * with the smallest row index if several do) the walk moves there, else it ends.  The emitted
+ * tokens are the target's own greedy continuation (lossless).  out_dev holds 2 + 3 * n_rows int32:
+ * [0] = number of tokens emitted (>= 1), [1] = number of leading rows of the accepted path that are
+ * the chain 0, 1, 2, .. and therefore already sit in the cache at their positions (>= 1: the root),
+ * [2 ..] the emitted tokens, [2 + n_rows ..] the rows of the accepted path (the rest is scratch). */
+csd_status csd_tree_accept_greedy(const float* target_logits_dev, const int32_t* tokens_dev, const int32_t* parent_host,
+                                  int n_rows, int vocab, int32_t* out_dev, void* stream);
+
 /* Prompt prefill: the model takes the input tokens in one run (Section 2).  Appends n tokens
  * (any n >= 1 with kv_len + n <= max_seq) at positions kv_len .. kv_len+n-1 to the cache of every
  * layer and produces no logits.  Models whose layer matrices are large enough for the tensor-core

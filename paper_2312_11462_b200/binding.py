@@ -77,6 +77,8 @@ lib.csd_model_destroy.argtypes = [_vp]
 lib.csd_encoder_forward.argtypes = [_vp, _vp, _i, _vp]
 lib.csd_review_forward.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
 lib.csd_prefill.argtypes = [_vp, _vp, _i, _i, _vp]
+lib.csd_review_forward_tree.argtypes = [_vp, _vp, _vp, _i, _i, _vp, _vp]
+lib.csd_tree_accept_greedy.argtypes = [_vp, _vp, _vp, _i, _i, _vp, _vp]
 lib.csd_model_profile.argtypes = [_vp, _i]
 lib.csd_model_profile_read.argtypes = [_vp, _vp, _vp]
 lib.csd_set_gemm_path.argtypes = [_i]
@@ -172,6 +174,17 @@ class Model:
                lib.csd_review_forward(self.h, _ptr(block_tokens), m, kv_len, _ptr(logits_out), _stream()))
         return logits_out
 
+    def csd_review_forward_tree(self, block_tokens: torch.Tensor, parent, kv_len: int) -> torch.Tensor:
+        """Logits [m, vocab] of a tree-shaped block; parent[r] < r is the row of r's parent, parent[0] = -1."""
+        assert block_tokens.dtype == torch.int32 and block_tokens.is_cuda
+        m = block_tokens.numel()
+        par = np.ascontiguousarray(np.asarray(parent, dtype=np.int32))
+        assert par.size == m
+        out = torch.empty(m, self.shape.vocab, dtype=torch.float32, device=block_tokens.device)
+        _check("csd_review_forward_tree",
+               lib.csd_review_forward_tree(self.h, _ptr(block_tokens), par.ctypes.data_as(_vp), m, kv_len, _ptr(out), _stream()))
+        return out
+
     def csd_prefill(self, tokens: torch.Tensor, kv_len: int) -> None:
         """Appends the tokens to the cache (wide blocks where the model allows them); no logits."""
         assert tokens.dtype == torch.int32 and tokens.is_cuda and tokens.is_contiguous()
@@ -210,6 +223,19 @@ def csd_linear(W: torch.Tensor, X: torch.Tensor, workspace: Optional[torch.Tenso
     _check("csd_linear", lib.csd_linear(_ptr(W), N, K, _ptr(X), m, _ptr(out), _ptr(workspace), workspace.numel(),
                                         _stream()))
     return out
+
+
+def csd_tree_accept_greedy(target_logits: torch.Tensor, tokens: torch.Tensor, parent):
+    """Returns (emitted tokens, rows of the accepted path, number of leading path rows valid in the cache)."""
+    m, V = target_logits.shape
+    assert target_logits.dtype == torch.float32 and target_logits.is_contiguous() and tokens.dtype == torch.int32
+    par = np.ascontiguousarray(np.asarray(parent, dtype=np.int32))
+    out = torch.zeros(2 + 3 * m, dtype=torch.int32, device=target_logits.device)
+    _check("csd_tree_accept_greedy",
+           lib.csd_tree_accept_greedy(_ptr(target_logits), _ptr(tokens), par.ctypes.data_as(_vp), m, V, _ptr(out), _stream()))
+    o = out.cpu().numpy()
+    n = int(o[0])
+    return o[2:2 + n].copy(), o[2 + m:2 + m + n].copy(), int(o[1])
 
 
 def csd_set_gemm_path(path: int) -> None:

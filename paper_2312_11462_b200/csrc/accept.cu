@@ -838,6 +838,94 @@ extern "C" csd_status csd_spec_accept(const float* target_logits_dev, const floa
                       seed, step, n_accepted_dev, out_token_dev, (char*)workspace_dev, L, status, (cudaStream_t)stream);
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// Greedy acceptance along a tree of drafted tokens (tree attention, Section 5.1 / Appendix B).
+// ---------------------------------------------------------------------------------------------
+namespace csd {
+
+struct TreeShape { int parent[CSD_MAX_ROWS]; };
+
+// arg-max of every row of the target logits (smallest index on ties), one CTA per row
+__global__ void __launch_bounds__(256)
+tree_argmax_kernel(const float* __restrict__ logits, int V, int* __restrict__ arg) {
+    pdl_wait();
+    pdl_trigger();
+    const float* x = logits + (size_t)blockIdx.x * V;
+    float best = -INFINITY;
+    int at = 0x7fffffff;
+    for (int i = threadIdx.x; i < V; i += 256) {
+        const float v = x[i];
+        if (v > best || at == 0x7fffffff) { best = v; at = i; }
+    }
+    __shared__ float s_v[256];
+    __shared__ int s_i[256];
+    s_v[threadIdx.x] = best; s_i[threadIdx.x] = at;
+    __syncthreads();
+    for (int o = 128; o > 0; o >>= 1) {
+        if (threadIdx.x < o) {
+            const float ov = s_v[threadIdx.x + o];
+            const int oi = s_i[threadIdx.x + o];
+            if (ov > s_v[threadIdx.x] || (ov == s_v[threadIdx.x] && oi < s_i[threadIdx.x])) { s_v[threadIdx.x] = ov; s_i[threadIdx.x] = oi; }
+        }
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) arg[blockIdx.x] = s_i[0] == 0x7fffffff ? 0 : s_i[0];
+}
+
+// out[0] = tokens emitted, out[1] = leading rows of the accepted path that are a chain 0, 1, 2, ..
+// (their cache entries are valid), out[2 ..] = the emitted tokens, out[2 + m ..] = rows of the path
+__global__ void tree_walk_kernel(const int* __restrict__ arg, const int* __restrict__ tokens, const TreeShape shape, int m,
+                                 int V, int* __restrict__ out, int* status) {
+    if (threadIdx.x != 0) return;
+    int cur = 0, n_out = 0, n_valid = 1;
+    bool chain = true;
+    out[2 + m] = 0;
+    while (true) {
+        const int y = arg[cur];
+        out[2 + n_out] = y;
+        ++n_out;
+        int nxt = -1;
+        for (int c = cur + 1; c < m; ++c) {
+            const int t = tokens[c];
+            if (t < 0 || t >= V) { set_status(status, CSD_ERR_BAD_TOKEN); continue; }
+            if (shape.parent[c] == cur && t == y) { nxt = c; break; }
+        }
+        if (nxt < 0 || n_out >= m) break;
+        out[2 + m + n_out] = nxt;
+        chain = chain && nxt == n_out;
+        if (chain) n_valid = n_out + 1;
+        cur = nxt;
+    }
+    out[0] = n_out;
+    out[1] = n_valid;
+}
+
+}  // namespace csd
+
+extern "C" csd_status csd_tree_accept_greedy(const float* target_logits_dev, const int32_t* tokens_dev,
+                                             const int32_t* parent_host, int n_rows, int V, int32_t* out_dev, void* stream) {
+    if (!target_logits_dev || !tokens_dev || !parent_host || !out_dev || n_rows < 1 || n_rows > CSD_MAX_ROWS || V < 1)
+        return CSD_ERR_INVALID_ARG;
+    TreeShape shape;
+    for (int r = 0; r < CSD_MAX_ROWS; ++r) shape.parent[r] = -2;
+    for (int r = 0; r < n_rows; ++r) {
+        const int p = parent_host[r];
+        if (r == 0 ? p != -1 : (p < 0 || p >= r)) return CSD_ERR_INVALID_ARG;
+        shape.parent[r] = p;
+    }
+    int* status = status_word_device();
+    if (!status) return CSD_ERR_CUDA;
+    cudaStream_t st = (cudaStream_t)stream;
+    int* arg = (int*)out_dev + 2 + 2 * n_rows;
+    PdlLaunch la(dim3((unsigned)n_rows), dim3(256), 0, st);
+    CSD_CUDA(cudaLaunchKernelEx(&la.cfg, tree_argmax_kernel, target_logits_dev, V, arg));
+    tree_walk_kernel<<<1, 32, 0, st>>>((const int*)arg, (const int*)tokens_dev, shape, n_rows, V, (int*)out_dev, status);
+    count_launch(2);
+    CSD_CUDA(cudaGetLastError());
+    return CSD_OK;
+}
+
 // ---------------------------------------------------------------------------------------------
 // Variant for callers that must not allocate: its scratch is a fixed array inside the library.
 // ---------------------------------------------------------------------------------------------

@@ -43,6 +43,11 @@ struct AttnParams {
     int* status;
     int ldq, ld_new, m, cap, H, n_keys, n_old, early_loads, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
+    // tree-shaped block: row r sees block row j only if bit j of tmask[r] is set (its ancestors and
+    // itself) and is rotated for position n_old + tdepth[r]; its cache slot stays n_old + r
+    int tree;
+    unsigned tmask[MAXM];
+    unsigned char tdepth[MAXM];
 };
 
 __device__ __forceinline__ void bulk_load(void* dst, const void* src, uint32_t bytes, uint64_t* bar) {
@@ -169,8 +174,9 @@ block_attention_kernel(const AttnParams p) {
     //      for the tiles that hold them and written to the cache by the CTA whose range they fall in
     for (int i = tid; i < m * half; i += AT) {
         const int r = i / half, d = i % half, pos = p.n_old + r;
+        const int rpos = p.n_old + (p.tree ? (int)p.tdepth[r] : r);      // position the rotation uses
         float c = 1.f, s = 0.f;
-        if (p.rope_cos) { c = p.rope_cos[(size_t)pos * half + d]; s = p.rope_sin[(size_t)pos * half + d]; }
+        if (p.rope_cos) { c = p.rope_cos[(size_t)rpos * half + d]; s = p.rope_sin[(size_t)rpos * half + d]; }
         const float* qr = p.q + (size_t)r * p.ldq + h * DH;
         const float q0 = qr[d], q1 = qr[d + half];
         const int e0 = d, e1 = d + half;
@@ -246,7 +252,9 @@ block_attention_kernel(const AttnParams p) {
                 if (part == 0) {
                     const int limit = p.causal ? p.n_keys + r : p.n_keys;   // keys [0, limit)
                     float s = -INFINITY;
-                    if (key < s_end && key < limit) {
+                    bool vis = key < s_end && key < limit;
+                    if (p.tree && key >= p.n_old) vis = key < s_end && ((p.tmask[r] >> (key - p.n_old)) & 1u);
+                    if (vis) {
                         s = d * p.scale;
                         if (bias_h) {
                             int bi = key - (p.q_pos0 + r) + p.bias_zero;
@@ -453,7 +461,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
         const int i = tid + e * AT;
         rc[e] = 1.f; rs[e] = 0.f;
         if (i < m * half && p.rope_cos) {
-            const size_t at = (size_t)(p.n_old + i / half) * half + i % half;
+            const size_t at = (size_t)(p.n_old + (p.tree ? (int)p.tdepth[i / half] : i / half)) * half + i % half;
             rc[e] = p.rope_cos[at]; rs[e] = p.rope_sin[at];
         }
     }
@@ -577,7 +585,9 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                     if (r < m) {
                         const int key = t0 + j, limit = p.causal ? p.n_keys + r : p.n_keys;
                         float s = -INFINITY;
-                        if (key < s_end && key < limit) {
+                        bool vis = key < s_end && key < limit;
+                        if (p.tree && key >= p.n_old) vis = key < s_end && ((p.tmask[r] >> (key - p.n_old)) & 1u);
+                        if (vis) {
                             s = sacc[mt][e] * p.scale;
                             if (bias_h) {
                                 int bi = key - (p.q_pos0 + r) + p.bias_zero;
@@ -775,6 +785,12 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     ap.early_loads = a.kv_settled ? 1 : 0;
     ap.causal = a.causal; ap.bias_len = a.bias_len; ap.bias_zero = a.bias_zero; ap.q_pos0 = a.q_pos0;
     ap.ldo = a.ldo; ap.scale = a.scale; ap.out_xs = a.out_xs; ap.out_xs_ld = a.out_xs_ld;
+    ap.tree = 0;
+    if (a.tree_mask) {
+        if (!append || !a.tree_depth || a.bias) return CSD_ERR_INVALID_ARG;
+        ap.tree = 1;
+        for (int r = 0; r < MAXM; ++r) { ap.tmask[r] = r < a.m ? a.tree_mask[r] : 0u; ap.tdepth[r] = r < a.m ? (unsigned char)a.tree_depth[r] : 0; }
+    }
     ap.nsplit = attn_splits(total, a.H);
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;

@@ -33,6 +33,11 @@ struct AttnArgs {
     // the kernel right before this one on the stream began; the tile requests then go out before
     // the dependency wait
     bool kv_settled = false;
+    // tree-shaped block (host arrays of m entries, copied into the launch): bit j of tree_mask[r] set
+    // when row r may see block row j; tree_depth[r] = number of ancestors of row r inside the block.
+    // Null: the block is a chain (row r sees rows 0..r).
+    const unsigned* tree_mask = nullptr;
+    const int* tree_depth = nullptr;
 };
 
 int attn_splits(int total_keys, int H);

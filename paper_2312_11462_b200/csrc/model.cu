@@ -673,8 +673,32 @@ extern "C" csd_status csd_prefill(csd_model* M, const int32_t* tokens_dev, int n
     return CSD_OK;
 }
 
+static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
+                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth);
+
 extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
                                          float* logits_out_dev, void* stream) {
+    return review_forward_impl(M, block_tokens_dev, m, kv_len, logits_out_dev, stream, nullptr, nullptr);
+}
+
+extern "C" csd_status csd_review_forward_tree(csd_model* M, const int32_t* block_tokens_dev, const int32_t* parent_host,
+                                              int m, int kv_len, float* logits_out_dev, void* stream) {
+    if (!M || !parent_host || m < 1 || m > CSD_MAX_ROWS) return CSD_ERR_INVALID_ARG;
+    if (M->cfg.arch != 0) return CSD_ERR_UNSUPPORTED;         // positions enter through the rotary embedding only
+    unsigned mask[CSD_MAX_ROWS];
+    int depth[CSD_MAX_ROWS];
+    for (int r = 0; r < m; ++r) {
+        const int p = parent_host[r];
+        if (r == 0 ? p != -1 : (p < 0 || p >= r)) return CSD_ERR_INVALID_ARG;   // row 0 is the root, parents come first
+        mask[r] = (r == 0 ? 0u : mask[p]) | (1u << r);
+        depth[r] = r == 0 ? 0 : depth[p] + 1;
+    }
+    if (kv_len + m > M->cfg.max_seq) return CSD_ERR_CAPACITY;
+    return review_forward_impl(M, block_tokens_dev, m, kv_len, logits_out_dev, stream, mask, depth);
+}
+
+static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
+                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth) {
     if (!M || !block_tokens_dev) return CSD_ERR_INVALID_ARG;
     const csd_model_config& c = M->cfg;
     if (m < 1 || m > c.max_rows || kv_len < 0) return CSD_ERR_INVALID_ARG;
@@ -710,6 +734,7 @@ extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_toke
         a.k_new = M->qkv + di; a.v_new = M->qkv + 2 * di; a.ld_new = 3 * di;
         a.kv_settled = true;      // committed rows date from earlier forwards
         if (c.arch == 0) { a.rope_cos = M->rope_c; a.rope_sin = M->rope_s; }
+        a.tree_mask = tree_mask; a.tree_depth = tree_depth;
         if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
         CSD_TRY(attention(M, a, st));
         // output projection into the residual rows; hands them on to the norm that follows
