@@ -120,6 +120,19 @@ csd_status csd_encoder_forward(csd_model* m, const int32_t* enc_tokens_dev, int 
 csd_status csd_review_forward(csd_model* m, const int32_t* block_tokens_dev, int n_rows, int kv_len,
                               float* logits_out_dev, void* stream);
 
+/* Batched review: the blocks of several sequences in one pass over the weights (the paper runs
+ * batch 1; with k+1 <= 5 rows per sequence three sequences still fit the 17 rows one pass takes,
+ * and the weights stream once for all of them).  models[0 .. n_seqs) are handles made from the SAME
+ * weights and the same configuration, each with its own workspace, i.e. its own cache (for arch 1
+ * each after its own csd_encoder_forward).  block_tokens_dev holds the sequences' rows one after
+ * the other (n_rows_host[g] rows of sequence g at positions kv_len_host[g] ..), logits_out_dev
+ * [sum of rows, vocab] in the same order (NULL: append only).  The contractions use the buffers of
+ * models[0]; every sequence's attention reads and appends its own cache.  Sum of rows <= max_rows.
+ * The host arrays are read before the call returns. */
+csd_status csd_review_forward_batch(csd_model* const* models, int n_seqs, const int32_t* block_tokens_dev,
+                                    const int32_t* n_rows_host, const int32_t* kv_len_host, float* logits_out_dev,
+                                    void* stream);
+
 /* Review of a TREE of drafted tokens in one pass (Section 5.1 and Appendix B combine the method
  * with tree attention: several candidate continuations hang off a node and the longest accepted
  * path wins).  Row 0 is the root (the newest token that is not in the cache yet, parent -1); row r

@@ -78,6 +78,7 @@ lib.csd_encoder_forward.argtypes = [_vp, _vp, _i, _vp]
 lib.csd_review_forward.argtypes = [_vp, _vp, _i, _i, _vp, _vp]
 lib.csd_prefill.argtypes = [_vp, _vp, _i, _i, _vp]
 lib.csd_review_forward_tree.argtypes = [_vp, _vp, _vp, _i, _i, _vp, _vp]
+lib.csd_review_forward_batch.argtypes = [_vp, _i, _vp, _vp, _vp, _vp, _vp]
 lib.csd_tree_accept_greedy.argtypes = [_vp, _vp, _vp, _i, _i, _vp, _vp]
 lib.csd_model_profile.argtypes = [_vp, _i]
 lib.csd_model_profile_read.argtypes = [_vp, _vp, _vp]
@@ -223,6 +224,25 @@ def csd_linear(W: torch.Tensor, X: torch.Tensor, workspace: Optional[torch.Tenso
     _check("csd_linear", lib.csd_linear(_ptr(W), N, K, _ptr(X), m, _ptr(out), _ptr(workspace), workspace.numel(),
                                         _stream()))
     return out
+
+
+def csd_review_forward_batch(models: Sequence["Model"], blocks: Sequence[torch.Tensor], kv_lens: Sequence[int],
+                             append_only: bool = False):
+    """One pass over the weights for the blocks of several sequences (models share weights and shape,
+    each has its own cache).  Returns the list of logits tensors, one per sequence."""
+    n = len(models)
+    rows = np.asarray([b_.numel() for b_ in blocks], dtype=np.int32)
+    kv = np.asarray(kv_lens, dtype=np.int32)
+    toks = torch.cat([b_.reshape(-1) for b_ in blocks]).contiguous()
+    assert toks.dtype == torch.int32 and toks.is_cuda
+    handles = (C.c_void_p * n)(*[m.h for m in models])
+    out = None if append_only else torch.empty(int(rows.sum()), models[0].shape.vocab, dtype=torch.float32, device=toks.device)
+    _check("csd_review_forward_batch",
+           lib.csd_review_forward_batch(handles, n, _ptr(toks), rows.ctypes.data_as(_vp), kv.ctypes.data_as(_vp),
+                                        _ptr(out), _stream()))
+    if out is None:
+        return None
+    return list(torch.split(out, [int(r) for r in rows]))
 
 
 def csd_tree_accept_greedy(target_logits: torch.Tensor, tokens: torch.Tensor, parent):

@@ -40,6 +40,7 @@ struct AttnParams {
     const float* q; const float* k_new; const float* v_new; const float* rope_cos; const float* rope_sin;
     __nv_bfloat16* Kc; __nv_bfloat16* Vc; const float* bias; float* out;
     __nv_bfloat16* out_xs; int out_xs_ld;
+    int xs_m, xs_r0;        // three-term output: rows per term of the whole buffer, row of this block's first row
     int* status;
     int ldq, ld_new, m, cap, H, n_keys, n_old, early_loads, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
@@ -101,9 +102,9 @@ __device__ __forceinline__ void merge_splits(cg::cluster_group& cluster, float* 
             uint16_t b1, b2, b3;
             split3(ov, b1, b2, b3);
             uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
-            xs[(size_t)r * p.out_xs_ld] = b1;
-            xs[(size_t)(m + r) * p.out_xs_ld] = b2;
-            xs[(size_t)(2 * m + r) * p.out_xs_ld] = b3;
+            xs[(size_t)(p.xs_r0 + r) * p.out_xs_ld] = b1;
+            xs[(size_t)(p.xs_m + p.xs_r0 + r) * p.out_xs_ld] = b2;
+            xs[(size_t)(2 * p.xs_m + p.xs_r0 + r) * p.out_xs_ld] = b3;
         }
     }
 }
@@ -330,7 +331,7 @@ block_attention_kernel(const AttnParams p) {
                 const float inv = row_l[r] > 0.f ? 1.f / row_l[r] : 0.f;
                 float* o = p.out + (size_t)r * p.ldo + h * DH + 2 * dp;
                 o[0] = acc[rr][0] * inv; o[1] = acc[rr][1] * inv;
-                if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, m, r, h * DH + 2 * dp, o[0], o[1]);
+                if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, p.xs_m, p.xs_r0 + r, h * DH + 2 * dp, o[0], o[1]);
             }
         }
         return;
@@ -677,7 +678,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                         const int d = 16 * warp + 8 * t + 2 * (lane & 3);
                         float* dst = p.out + (size_t)r * p.ldo + h * DH + d;
                         dst[0] = o[mt][t][2 * hr] * inv; dst[1] = o[mt][t][2 * hr + 1] * inv;
-                        if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, m, r, h * DH + d, dst[0], dst[1]);
+                        if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, p.xs_m, p.xs_r0 + r, h * DH + d, dst[0], dst[1]);
                     }
                 }
         }
@@ -785,6 +786,7 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     ap.early_loads = a.kv_settled ? 1 : 0;
     ap.causal = a.causal; ap.bias_len = a.bias_len; ap.bias_zero = a.bias_zero; ap.q_pos0 = a.q_pos0;
     ap.ldo = a.ldo; ap.scale = a.scale; ap.out_xs = a.out_xs; ap.out_xs_ld = a.out_xs_ld;
+    ap.xs_m = a.out_xs_rows > 0 ? a.out_xs_rows : a.m; ap.xs_r0 = a.out_xs_row0;
     ap.tree = 0;
     if (a.tree_mask) {
         if (!append || !a.tree_depth || a.bias) return CSD_ERR_INVALID_ARG;

@@ -20,6 +20,8 @@ struct AttnArgs {
     int ldo = 0;
     __nv_bfloat16* out_xs = nullptr;      // optional: the output rows as three bf16 terms, row = term * m + r
     int out_xs_ld = 0;
+    int out_xs_rows = 0;                  // rows per term of the out_xs buffer (0: m) and this block's first row in it
+    int out_xs_row0 = 0;
     // Self-attention of a drafted block (causal, n_keys = committed keys + 1): the block's own key
     // and value rows are still fp32 projections [m, ld_new]; the kernel rotates q and k (when
     // rope tables [pos][Dh/2] are given), rounds k and v to bf16, appends them to the cache at

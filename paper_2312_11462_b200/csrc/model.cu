@@ -673,12 +673,42 @@ extern "C" csd_status csd_prefill(csd_model* M, const int32_t* tokens_dev, int n
     return CSD_OK;
 }
 
+// A block may hold the rows of several sequences (batched review): the contractions run once over
+// all rows, the attention per sequence over that sequence's own cache.
+struct Segment { csd_model* S; int row0, rows, kv_len; };
 static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
-                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth);
+                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth,
+                                      const Segment* segs = nullptr, int nseg = 0);
 
 extern "C" csd_status csd_review_forward(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
                                          float* logits_out_dev, void* stream) {
     return review_forward_impl(M, block_tokens_dev, m, kv_len, logits_out_dev, stream, nullptr, nullptr);
+}
+
+extern "C" csd_status csd_review_forward_batch(csd_model* const* models, int n_seqs, const int32_t* block_tokens_dev,
+                                               const int32_t* n_rows_host, const int32_t* kv_len_host,
+                                               float* logits_out_dev, void* stream) {
+    if (!models || n_seqs < 1 || n_seqs > CSD_MAX_ROWS || !block_tokens_dev || !n_rows_host || !kv_len_host)
+        return CSD_ERR_INVALID_ARG;
+    csd_model* M = models[0];
+    if (!M) return CSD_ERR_INVALID_ARG;
+    Segment segs[CSD_MAX_ROWS];
+    int total = 0;
+    for (int g = 0; g < n_seqs; ++g) {
+        csd_model* S = models[g];
+        // one set of weights, one shape: the handles differ in their caches only
+        if (!S || S->embed != M->embed || memcmp(&S->cfg, &M->cfg, sizeof(M->cfg)) != 0) return CSD_ERR_INVALID_ARG;
+        for (int h = 0; h < g; ++h)
+            if (models[h] == S) return CSD_ERR_INVALID_ARG;
+        const int rows = n_rows_host[g], kv = kv_len_host[g];
+        if (rows < 1 || kv < 0) return CSD_ERR_INVALID_ARG;
+        if (kv + rows > M->cfg.max_seq) return CSD_ERR_CAPACITY;
+        if (M->cfg.arch == 1 && S->enc_len < 1) return CSD_ERR_INVALID_ARG;
+        segs[g] = Segment{S, total, rows, kv};
+        total += rows;
+    }
+    if (total > M->cfg.max_rows) return CSD_ERR_INVALID_ARG;
+    return review_forward_impl(M, block_tokens_dev, total, segs[0].kv_len, logits_out_dev, stream, nullptr, nullptr, segs, n_seqs);
 }
 
 extern "C" csd_status csd_review_forward_tree(csd_model* M, const int32_t* block_tokens_dev, const int32_t* parent_host,
@@ -698,8 +728,11 @@ extern "C" csd_status csd_review_forward_tree(csd_model* M, const int32_t* block
 }
 
 static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_dev, int m, int kv_len,
-                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth) {
+                                      float* logits_out_dev, void* stream, const unsigned* tree_mask, const int* tree_depth,
+                                      const Segment* segs, int nseg) {
     if (!M || !block_tokens_dev) return CSD_ERR_INVALID_ARG;
+    const Segment whole{M, 0, m, kv_len};
+    if (!segs) { segs = &whole; nseg = 1; }
     const csd_model_config& c = M->cfg;
     if (m < 1 || m > c.max_rows || kv_len < 0) return CSD_ERR_INVALID_ARG;
     if (kv_len + m > c.max_seq) return CSD_ERR_CAPACITY;
@@ -725,18 +758,23 @@ static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_
             if (x_ready) { qo.xs_in = M->xs_x; qo.ssq_in = M->ssq_x; qo.ssq_cnt = M->ssq_x_cnt; }
             CSD_TRY(project_qkv(M, y, M->x, m, M->qkv, st, &qo));
         }
-        AttnArgs a;
-        a.q = M->qkv; a.ldq = 3 * di; a.m = m; a.Kc = Kl; a.Vc = Vl; a.cap = c.max_seq; a.H = H; a.Dh = Dh;
-        a.n_keys = kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
-        if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = kv_len; }
-        a.out = M->attn; a.ldo = di;
-        // the block's own k and v rows go into the cache inside the attention kernel
-        a.k_new = M->qkv + di; a.v_new = M->qkv + 2 * di; a.ld_new = 3 * di;
-        a.kv_settled = true;      // committed rows date from earlier forwards
-        if (c.arch == 0) { a.rope_cos = M->rope_c; a.rope_sin = M->rope_s; }
-        a.tree_mask = tree_mask; a.tree_depth = tree_depth;
-        if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; }
-        CSD_TRY(attention(M, a, st));
+        for (int g = 0; g < nseg; ++g) {
+            const Segment& sg = segs[g];
+            AttnArgs a;
+            a.q = M->qkv + (size_t)sg.row0 * 3 * di; a.ldq = 3 * di; a.m = sg.rows;
+            a.Kc = sg.S->kcache + (size_t)l * sg.S->layer_kv; a.Vc = sg.S->vcache + (size_t)l * sg.S->layer_kv;
+            a.cap = c.max_seq; a.H = H; a.Dh = Dh;
+            a.n_keys = sg.kv_len + 1; a.causal = 1; a.scale = c.arch == 0 ? 1.f / sqrtf((float)Dh) : 1.f;
+            if (c.arch == 1) { a.bias = M->dec_bias; a.bias_len = c.max_seq; a.bias_zero = c.max_seq - 1; a.q_pos0 = sg.kv_len; }
+            a.out = M->attn + (size_t)sg.row0 * di; a.ldo = di;
+            // the block's own k and v rows go into the cache inside the attention kernel
+            a.k_new = a.q + di; a.v_new = a.q + 2 * di; a.ld_new = 3 * di;
+            a.kv_settled = true;      // committed rows date from earlier forwards
+            if (c.arch == 0) { a.rope_cos = M->rope_c; a.rope_sin = M->rope_s; }
+            a.tree_mask = tree_mask; a.tree_depth = tree_depth;
+            if (tc_o) { a.out_xs = M->xs_attn; a.out_xs_ld = di; a.out_xs_rows = m; a.out_xs_row0 = sg.row0; }
+            CSD_TRY(attention(M, a, st));
+        }
         // output projection into the residual rows; hands them on to the norm that follows
         LinOpt oo;
         if (tc_o) oo.xs_in = M->xs_attn;
@@ -748,13 +786,17 @@ static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_
             LinOpt xq;
             if (x_ready) { xq.xs_in = M->xs_x; xq.ssq_in = M->ssq_x; xq.ssq_cnt = M->ssq_x_cnt; }
             CSD_TRY(linear(M, y.xq, nullptr, di, d, M->x, d, m, y.norm_x, M->qkv, 3 * di, EPI_STORE, st, &xq));
-            AttnArgs x;
-            x.q = M->qkv; x.ldq = 3 * di; x.m = m; x.Kc = M->xk + (size_t)l * M->layer_x;
-            x.Vc = M->xv + (size_t)l * M->layer_x; x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = M->enc_len;
-            x.causal = 0; x.scale = 1.f; x.out = M->attn; x.ldo = di;
-            x.kv_settled = true;  // written once by the encoder pass
-            if (tc_o) { x.out_xs = M->xs_attn; x.out_xs_ld = di; }
-            CSD_TRY(attention(M, x, st));
+            for (int g = 0; g < nseg; ++g) {
+                const Segment& sg = segs[g];
+                AttnArgs x;
+                x.q = M->qkv + (size_t)sg.row0 * 3 * di; x.ldq = 3 * di; x.m = sg.rows;
+                x.Kc = sg.S->xk + (size_t)l * sg.S->layer_x; x.Vc = sg.S->xv + (size_t)l * sg.S->layer_x;
+                x.cap = c.max_enc_len; x.H = H; x.Dh = Dh; x.n_keys = sg.S->enc_len;
+                x.causal = 0; x.scale = 1.f; x.out = M->attn + (size_t)sg.row0 * di; x.ldo = di;
+                x.kv_settled = true;  // written once by the encoder pass
+                if (tc_o) { x.out_xs = M->xs_attn; x.out_xs_ld = di; x.out_xs_rows = m; x.out_xs_row0 = sg.row0; }
+                CSD_TRY(attention(M, x, st));
+            }
             LinOpt xo;
             if (tc_o) xo.xs_in = M->xs_attn;
             x_ready = tc_o && linear_uses_tensor_cores(m, ff, d, true);
