@@ -10,8 +10,8 @@
 // K block rides in the same stage as the weight tile; the epilogue adds the three partial results.
 //
 // Work is cut into (tile, K block) units and every CTA (one per SM) owns an equal contiguous share
-// of them, so all SMs stream the same number of bytes; a tile that straddles two CTAs is finished
-// by whichever of them arrives last at the tile's ticket, adding the parts in CTA order
+// of them, so all SMs stream the same number of bytes; a tile that straddles CTAs is finished by
+// the first of them (for which it comes last), adding the parts the others parked in CTA order
 // (deterministic).  Roles inside a CTA (192 threads): warp 0 lane 0 issues TMA, warp 1 lane 0
 // issues MMA, warps 2-5 read the accumulators from tensor memory (one quadrant each) and run the
 // epilogue: rms-norm factor, residual add or gated activation, and optionally the three-term
@@ -160,7 +160,7 @@ struct __align__(8) TcCtrl {
     uint64_t full[12], empty[12], acc_full[2], acc_empty[2];
     uint64_t red_ready, red_done;      // cluster split: the leader's buffer is free / all parts have been written
     uint32_t tmem_base;
-    int abort_flag, last_flag;
+    int abort_flag;
     float scale[32];
 };
 
@@ -204,6 +204,12 @@ __device__ __forceinline__ bool mbar_wait_cluster(uint64_t* bar, uint32_t parity
     return false;
 }
 
+__device__ __forceinline__ unsigned ld_acquire_gpu(const unsigned* p) {
+    unsigned v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+
 template <int M, bool DUAL>
 __global__ void __launch_bounds__(TC_THREADS, 2)
 skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_constant__ CUtensorMap tmW2,
@@ -240,7 +246,7 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
         for (int b = 0; b < 2; ++b) { mbar_init(&ctl->acc_full[b], 1); mbar_init(&ctl->acc_empty[b], 4); }
         mbar_init(&ctl->red_ready, 1);
         mbar_init(&ctl->red_done, 4 * 3);               // one arrival per epilogue warp of the three other CTAs
-        ctl->abort_flag = 0; ctl->last_flag = 0;
+        ctl->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     }
     if (warp == 1) {
@@ -427,40 +433,46 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                     continue;
                 }
             } else if (seg_len < p.nkb) {
-                // part of a tile: leave it in this CTA's slot (0 = the CTA's first segment, 1 = a later
-                // one); the CTA that arrives last adds all parts in CTA order and finishes the tile
-                float* mine = my_part + (size_t)(seg == 0 ? 0 : 1) * NT * M * TILE_N;
-#pragma unroll
-                for (int u = 0; u < NT; ++u)
-#pragma unroll
-                    for (int r = 0; r < M; ++r) mine[(u * M + r) * TILE_N + col] = sums[u][r];
-                __threadfence();
-                asm volatile("bar.sync 1, 128;" ::: "memory");
+                // Part of a tile.  Its contributors are consecutive CTAs; the first of them finishes it.
+                // For the last contributor the tile is the FIRST thing it computes, so its partial sums
+                // are parked in global memory (and its arrival counted) long before the first contributor,
+                // for which the tile comes LAST, asks for them; a contributor whose whole share lies inside
+                // the tile parks at the end, and the finisher waits for it (bounded).  Parts are added in
+                // CTA order (deterministic).  Measured against "whoever arrives last finishes": 1.7 % faster
+                // per forward at 5 rows, 4 % at 17; taking the first contributor's part of the tile first,
+                // so that a middle contributor can finish without waiting, was slower again.
                 const int c_lo = cta_of_unit((unsigned)tile * p.nkb, units, ctas);
                 const int c_hi = cta_of_unit((unsigned)(tile + 1) * p.nkb - 1, units, ctas);
+                if (cta != c_lo) {
+                    float* mine = my_part;              // (a later contributor's part opens its share: slot 0)
+#pragma unroll
+                    for (int u = 0; u < NT; ++u)
+#pragma unroll
+                        for (int r = 0; r < M; ++r) mine[(u * M + r) * TILE_N + col] = sums[u][r];
+                    __threadfence();
+                    asm volatile("bar.sync 1, 128;" ::: "memory");
+                    if (et == 0) atomicAdd(&p.tickets[tile], 1u);
+                    continue;
+                }
                 if (et == 0) {
-                    const unsigned old = atomicAdd(&p.tickets[tile], 1u);
-                    ctl->last_flag = (old == (unsigned)(c_hi - c_lo));
-                    if (ctl->last_flag) p.tickets[tile] = 0u;
+                    const unsigned want = (unsigned)(c_hi - c_lo);
+                    int spins = 0;
+                    while (ld_acquire_gpu(&p.tickets[tile]) < want) {
+                        if (++spins > SPIN_LIMIT) { *abort_flag = 1; break; }
+                    }
+                    p.tickets[tile] = 0u;               // everyone has arrived: ready for the next launch
                 }
                 asm volatile("bar.sync 1, 128;" ::: "memory");
-                const int last = ctl->last_flag;        // (rewritten only after every warp has passed the next bar.sync)
-                if (!last) continue;
                 __threadfence();
-#pragma unroll
-                for (int u = 0; u < NT; ++u)
-#pragma unroll
-                    for (int r = 0; r < M; ++r) sums[u][r] = 0.f;
-                // parts in CTA order; as many contributors' loads in flight together as about 48 registers
-                // hold (all of them, in one round trip, for a 5-row block)
+                // the other parts in CTA order; as many contributors' loads in flight together as about 48
+                // registers hold (all of them, in one round trip, for a 5-row block)
                 constexpr int NV = NT * M, CH = NV <= 6 ? 8 : (48 / NV < 1 ? 1 : 48 / NV);
-                for (int c = c_lo; c <= c_hi; c += CH) {
+                for (int c = c_lo + 1; c <= c_hi; c += CH) {
                     float part[CH][NV];
 #pragma unroll
                     for (int h = 0; h < CH; ++h) {
                         const int cc = min(c + h, c_hi);
-                        const int slot = (int)(unit_begin(cc, units, ctas) / p.nkb) == tile ? 0 : 1;
-                        const float* src = p.partial + ((size_t)cc * 2 + slot) * NT * M * TILE_N + col;
+                        const float* src = p.partial + ((size_t)cc * 2) * NT * M * TILE_N + col;
 #pragma unroll
                         for (int v = 0; v < NV; ++v) part[h][v] = __ldcg(src + v * TILE_N);
                     }
