@@ -31,7 +31,7 @@ PROMPT_LEN, MAX_NEW, MAX_BLOCK = 128, 256, 4
 K_MATRIX = [[4, 0], [0, 4]]
 WORKLOAD = "llama7b-shaped target + 68M-shaped draft + Max-Gram, prompt 128, generate 256, greedy, K=[[4,0],[0,4]]"
 METRIC = "generated tokens/s and review-step HBM GB/s (% of 8 TB/s) at 1 B200"
-TRAFFIC_RATIO = 1.039                  # DRAM bytes / weight bytes of the tensor-core GEMM, from its ncu capture
+TRAFFIC_RATIO = 1.038                  # DRAM bytes / weight bytes of the tensor-core GEMM, from its ncu capture
 ORACLE_PROMPT, ORACLE_NEW = 8, 4       # bounded CPU sample: same models, 8-token prompt, 4 new tokens
 
 
@@ -252,10 +252,17 @@ def run_ours(args):
     roofline = {"bound": "hbm", "kernel": "skinny_gemm_tc_kernel (TMA-staged weight-streaming GEMM on tcgen05, m=5)", "achieved": gemm_gbs,
                 "peak": peak, "peak_kind": f"{peak_kind} STREAM-style copy", "unit": "GB/s", "frac": gemm_gbs / peak,
                 "traffic": TRAFFIC_RATIO * prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
-                "traffic_note": "dram read+write per launch = algorithmic bytes x 1.039, the ratio ncu measured on "
-                                "the o / gate+up / down launches of one layer (profiles/skinny_gemm_tc_kernel_*)",
+                "traffic_note": "dram read+write per launch = algorithmic bytes x 1.038, the ratio ncu measured over "
+                                "the q|k|v / o / gate+up / down launches of one layer (profiles/skinny_gemm_tc_kernel_*)",
                 "bytes_per_launch": prof["gemm_weight_bytes"] / max(prof["gemm_launches"], 1),
                 "us_per_launch": gemm_launch_us}
+    # the same kernel inside the pipelined forward (no event between launches, so the next launch's prologue
+    # overlaps the tail of this one): the timed review forward apportioned by the bracketed shares
+    class_ms = prof["gemm_ms"] + prof["attn_ms"] + prof["other_ms"]
+    piped_us = review_us * prof["gemm_ms"] / class_ms
+    piped_gbs = weight_bytes / piped_us / 1e3
+    roofline["in_pipeline"] = {"us_per_forward": piped_us, "achieved": piped_gbs, "frac": piped_gbs / peak,
+                               "note": "review forward timed as a whole x the GEMM's share of the bracketed launches"}
 
     # every kernel class of the review step against its own HBM roofline (event pairs around each launch,
     # so consecutive kernels do not overlap here as they do in the timed forward)
@@ -281,7 +288,7 @@ def run_ours(args):
     other = None
     if world == 1 and not args.no_configs:
         draft.close()
-        other = {"tiny_cascade": cfg_tiny(b),
+        other = {"variants": cfg_variants(b, ts, tb, target, prompt), "tiny_cascade": cfg_tiny(b),
                  "accept": [cfg_accept(b, peak, 128256, 16, 0.5), cfg_accept(b, peak, 128256, 4, 0.5),
                             cfg_accept(b, peak, 32000, 4, 0.5)],
                  "long_cache_review_step": cfg_long(b, peak, tb, reviews=6)}
@@ -321,21 +328,26 @@ def run_review_only(args):
     import workloads
     from dataclasses import replace
     from paper_2312_11462_b200 import binding as b
-    ts = workloads.SHAPES["llama7b"]
+    if args.accept_only:
+        V, k = (int(x) for x in args.accept_only.split(","))
+        peak, _ = measured_peaks()
+        print(json.dumps(cfg_accept(b, peak, V, k, 0.5)), flush=True)
+        return
+    S = args.cache or PROMPT_LEN
+    ts = workloads.SHAPES["llama7b" if S + 32 <= workloads.SHAPES["llama7b"].max_seq else "llama7b_long"]
     if args.layers:
         ts = replace(ts, n_layers=args.layers)
     tb = workloads.make_weights(ts, seed=100, device="cuda")
-    prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, PROMPT_LEN + MAX_BLOCK + 1, seed=1000)).cuda()
+    prompt = torch.from_numpy(workloads.make_prompt(ts.vocab, S + MAX_BLOCK + 1, seed=1000)).cuda()
     target = b.Model(ts, tb)
-    for p0 in range(0, PROMPT_LEN, 16):
-        target.csd_review_forward(prompt[p0:p0 + 16], p0)
-    blk = prompt[PROMPT_LEN:PROMPT_LEN + MAX_BLOCK + 1].contiguous()
+    target.csd_prefill(prompt[:S].contiguous(), 0)              # wide passes of 128 rows
+    blk = prompt[S:S + MAX_BLOCK + 1].contiguous()
     logits = torch.empty(MAX_BLOCK + 1, ts.vocab, device="cuda")
     ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     torch.cuda.synchronize()
     ev0.record()
     for _ in range(args.review_only):
-        target.csd_review_forward(blk, PROMPT_LEN, logits)
+        target.csd_review_forward(blk, S, logits)
     ev1.record()
     torch.cuda.synchronize()
     tok = blk[:MAX_BLOCK].reshape(1, MAX_BLOCK).contiguous()
@@ -460,6 +472,37 @@ def cfg_long(b, peak, tb, block_rows=(2, 5, 9, 17), reviews=8, S=2048):
     return out
 
 
+def cfg_variants(b, ts, tb, target, prompt):
+    """Review-step variants on the 7B-shaped target: a tree-shaped block (the paper's tree-attention
+    setting: eight candidates at the first position, the lead continued by a chain of three) and a
+    batched review (three sequences of five rows in one pass over the weights)."""
+    import torch
+    parent = [-1] + [0] * 8 + [1, 9, 10]
+    toks = torch.from_numpy(prompt[:len(parent)].copy()).cuda()
+    for _ in range(3):
+        lg = target.csd_review_forward_tree(toks, parent, PROMPT_LEN)
+    out = torch.zeros(2 + 3 * len(parent), dtype=torch.int32, device="cuda")
+    par = np.asarray(parent, dtype=np.int32)
+
+    def tree_step(i):
+        lg = target.csd_review_forward_tree(toks, parent, PROMPT_LEN)
+        b._check("csd_tree_accept_greedy", b.lib.csd_tree_accept_greedy(lg.data_ptr(), toks.data_ptr(), par.ctypes.data, len(parent),
+                                                                      ts.vocab, out.data_ptr(), b._stream()))
+    tree_us = timed_us(tree_step, 10)
+    others = [b.Model(ts, tb) for _ in range(2)]
+    models = [target] + others
+    blocks = [torch.from_numpy(prompt[i:i + MAX_BLOCK + 1].copy()).cuda() for i in range(3)]
+    for m_ in others:
+        m_.csd_prefill(torch.from_numpy(prompt[:PROMPT_LEN].copy()).cuda(), 0)
+    for _ in range(3):
+        b.csd_review_forward_batch(models, blocks, [PROMPT_LEN] * 3)
+    batch_us = timed_us(lambda i: b.csd_review_forward_batch(models, blocks, [PROMPT_LEN] * 3), 10)
+    for m_ in others:
+        m_.close()
+    return {"tree_review_step": {"rows": len(parent), "shape": "8 candidates at the first position, lead + chain of 3", "us": tree_us},
+            "batched_review": {"sequences": 3, "rows_each": MAX_BLOCK + 1, "us": batch_us, "us_per_sequence": batch_us / 3}}
+
+
 def cfg_t5(b, cascade=True):
     """Configuration 4: T5-xxl-shaped target with base- and small-shaped drafts, temperature 1."""
     import torch
@@ -533,11 +576,13 @@ def main():
     ap.add_argument("--no-configs", action="store_true", help="leave the samples of the other configurations out of the line")
     ap.add_argument("--review-only", type=int, default=0, help="profiling aid: only N review forwards of the target")
     ap.add_argument("--layers", type=int, default=0, help="with --review-only: cut the target to L layers")
+    ap.add_argument("--cache", type=int, default=0, help="with --review-only: committed cache length (default 128)")
+    ap.add_argument("--accept-only", default="", help="profiling aid: V,k of one 64-row accept case (sigma 0.5), timed alone")
     ap.add_argument("--configs", default="", help="measure other configurations: tiny,accept,long,t5")
     args = ap.parse_args()
     if args.configs:
         run_configs(args)
-    elif args.review_only:
+    elif args.review_only or args.accept_only:
         run_review_only(args)
     elif args.impl == "reference":
         run_reference(args)
