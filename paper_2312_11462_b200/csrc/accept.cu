@@ -509,8 +509,8 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
 // ---------------------------------------------------------------------------------------------
 // resample, one kernel: a row is a thread-block cluster of up to RF_MAXC CTAs; a CTA keeps its
 // slice of the two logit vectors (position n only) in registers, so global memory is read once.
-// Round 1: per-CTA sums of the exponentials, exchanged through distributed shared memory -> the
-// normalisers.  Round 2: per-CTA residual mass -> total mass S and the CTA whose slice holds
+// First exchange: per-CTA sums of the exponentials, exchanged through distributed shared memory -> the
+// normalisers.  Second exchange: per-CTA residual mass -> total mass S and the CTA whose slice holds
 // u2 * S.  That CTA scans its threads' sums in thread order and picks the entry.  All sums have a
 // fixed order (lanes by xor-shuffle or prefix scan, warps and CTAs in index order).
 // ---------------------------------------------------------------------------------------------
@@ -593,7 +593,7 @@ resample_fused_kernel(const float* __restrict__ tl, const float* __restrict__ dl
             sq += ed[j + i];
         }
     }
-    // ---- round 1: normalisers
+    // ---- first exchange: normalisers
     sp = rf_block_sum(sp, s_warp);
     sq = rf_block_sum(sq, s_warp);
     if (threadIdx.x == 0) { s_ex[0] = sp; s_ex[1] = sq; }
@@ -612,7 +612,7 @@ resample_fused_kernel(const float* __restrict__ tl, const float* __restrict__ dl
         const double r = p - q;
         return r > 0.0 ? r : 0.0;
     };
-    // ---- round 2: masses (a second time with the target law itself if the residual is empty)
+    // ---- second exchange: masses (a second time with the target law itself if the residual is empty)
     int mode = ri.mode;
     double local = 0.0, S = 0.0, base = 0.0, my_mass = 0.0;
     int pick_cta = -1, last_pos = 0;

@@ -13,8 +13,8 @@ pytestmark = pytest.mark.gpu
 
 @pytest.fixture(scope="module", params=[0, 1, 2, 3], ids=["automatic", "cuda-core", "tensor-core", "tensor-core-row-ranges"])
 def b(request):
-    """Every test here runs once per kernel family: the automatic choice (small models go through the
-    whole-forward kernel), CUDA-core GEMM (128-bit loads + fp32 FMA) with the CUDA-core attention, and
+    """Every test here runs once per kernel family: the automatic choice (small matrices go through the
+    CUDA-core kernel), CUDA-core GEMM (128-bit loads + fp32 FMA) with the CUDA-core attention, and
     the two tensor-core GEMMs (TMA + tcgen05) with the tensor-core attention."""
     require_gpu()
     from paper_2312_11462_b200 import binding

@@ -91,6 +91,30 @@ def long_cache_review_blocks(b, orc):
     assert b.csd_device_status() == 0
 
 
+@pytest.mark.parametrize("d_head,n_heads", [(64, 48), (128, 40)])
+def test_long_cache_many_heads(b, orc, d_head, n_heads):
+    """Long caches at both tensor-core head dimensions with 40 and 48 heads: every CTA walks more
+    tiles than its ring holds, so ring slots are refilled; cache lengths before, on and after a
+    tile edge, blocks of one and two row tiles; the cache comes from a wide-block prefill."""
+    shape = llama_shape(1, d_head * n_heads, n_heads, 1024, 1000, 2300)
+    blob = workloads.make_weights(shape, seed=33, device="cuda", std=0.03, gain_std=0.2)
+    toks = workloads.make_prompt(shape.vocab, 2300, seed=8)
+    gm, om = b.Model(shape, blob), orc.Model(shape, orc.blob_to_u16(blob))
+    S = 2040
+    for pos in range(0, S, 510):
+        om.review_forward(toks[pos:pos + 510], pos)
+    gm.csd_prefill(to_dev_i32(toks[:S]), 0)
+    pos = S
+    for m in (5, 3, 17, 9, 16, 17, 1, 12):      # 2040, 2045, 2048, 2065, 2074, 2090, 2107, 2108
+        blk = toks[pos:pos + m]
+        g = gm.csd_review_forward(to_dev_i32(blk), pos).cpu().numpy()
+        r = om.review_forward(blk, pos)
+        assert rel_l2(g, r) <= LOGIT_REL_L2, (pos, m, rel_l2(g, r))
+        assert np.abs(g - r).max() <= LOGIT_MAX_ABS
+        pos += m
+    assert b.csd_device_status() == 0
+
+
 def sub_stack(shape, blob, n_layers):
     """The first n_layers decoder layers of a blob (with its embedding, final norm and head)."""
     from dataclasses import replace
