@@ -42,6 +42,7 @@ struct AttnParams {
     __nv_bfloat16* out_xs; int out_xs_ld;
     int xs_m, xs_r0;        // three-term output: rows per term of the whole buffer, row of this block's first row
     int* status;
+    int sub_rows;           // > 0: grid.z sub-blocks of this many rows each, over a cache that already holds every row
     int ldq, ld_new, m, cap, H, n_keys, n_old, early_loads, causal, bias_len, bias_zero, q_pos0, ldo, nsplit, split_len;
     float scale;
     // tree-shaped block: row r sees block row j only if bit j of tmask[r] is set (its ancestors and
@@ -72,8 +73,9 @@ __device__ __forceinline__ void store_split(__nv_bfloat16* xs, int ld, int m, in
 // distributed shared memory: the CTAs of a head share out the m*DH output elements; each thread
 // first fetches everything it needs from all splits in one batch of independent remote loads.
 template <int DH, int REC>
-__device__ __forceinline__ void merge_splits(cg::cluster_group& cluster, float* rec, const AttnParams& p, int h, int split) {
-    const int m = p.m;
+__device__ __forceinline__ void merge_splits(cg::cluster_group& cluster, float* rec, const AttnParams& p, int h, int split,
+                                             int m, int r0) {
+    // m rows of this CTA's records; they are rows r0 .. r0+m-1 of the launch's output
     for (int i = split * AT + threadIdx.x; i < m * DH; i += p.nsplit * AT) {
         const int r = i / DH, d = i % DH;
         float ms[MAX_SPLITS], ls[MAX_SPLITS], vs[MAX_SPLITS];
@@ -97,14 +99,14 @@ __device__ __forceinline__ void merge_splits(cg::cluster_group& cluster, float* 
                 den = fmaf(ls[s], w, den);
             }
         const float ov = den > 0.f ? num / den : 0.f;
-        p.out[(size_t)r * p.ldo + h * DH + d] = ov;
+        p.out[(size_t)(r0 + r) * p.ldo + h * DH + d] = ov;
         if (p.out_xs) {
             uint16_t b1, b2, b3;
             split3(ov, b1, b2, b3);
             uint16_t* xs = reinterpret_cast<uint16_t*>(p.out_xs) + h * DH + d;
-            xs[(size_t)(p.xs_r0 + r) * p.out_xs_ld] = b1;
-            xs[(size_t)(p.xs_m + p.xs_r0 + r) * p.out_xs_ld] = b2;
-            xs[(size_t)(2 * p.xs_m + p.xs_r0 + r) * p.out_xs_ld] = b3;
+            xs[(size_t)(p.xs_r0 + r0 + r) * p.out_xs_ld] = b1;
+            xs[(size_t)(p.xs_m + p.xs_r0 + r0 + r) * p.out_xs_ld] = b2;
+            xs[(size_t)(2 * p.xs_m + p.xs_r0 + r0 + r) * p.out_xs_ld] = b3;
         }
     }
 }
@@ -349,7 +351,7 @@ block_attention_kernel(const AttnParams p) {
     }
     if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
     cluster.sync();
-    merge_splits<DH, C::REC>(cluster, rec, p, h, split);
+    merge_splits<DH, C::REC>(cluster, rec, p, h, split, m, 0);
     cluster.sync();       // no CTA leaves while another may still read its record
 }
 
@@ -423,8 +425,12 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     cg::cluster_group cluster = cg::this_cluster();
     const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
     const int h = blockIdx.x, split = blockIdx.y;
-    const int m = p.m, half = DH / 2;
-    const int total = p.causal ? p.n_keys + m - 1 : p.n_keys;
+    // sub-block mode (sub_rows > 0, no append): blockIdx.z picks rows r0 .. r0+m-1 of a block of p.m rows
+    const int r0 = p.sub_rows ? (int)blockIdx.z * p.sub_rows : 0;
+    const int m = p.sub_rows ? min(p.sub_rows, p.m - r0) : p.m, half = DH / 2;
+    const int n_keys = p.n_keys + (p.causal ? r0 : 0);          // keys visible to this CTA's first row
+    const int total = p.causal ? n_keys + m - 1 : n_keys;
+    const int n_old = p.sub_rows ? total : p.n_old;
     const int s_begin = split * p.split_len;
     const int s_end = min(total, s_begin + p.split_len);
     const int n_tiles = s_end > s_begin ? (s_end - s_begin + TILE - 1) / TILE : 0;
@@ -455,14 +461,14 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     if (tid == 0 && p.early_loads)
         for (int it = 0; it < n_tiles && it < STAGES; ++it) request(it);
     // this thread's (row, dimension pair) items of the block; their rotation factors are constants
-    constexpr int ITEMS = (MAXM * (DH / 2) + AT - 1) / AT;
+    constexpr int ITEMS = ((R < MAXM ? R : (MT == 2 ? R : MAXM)) * (DH / 2) + AT - 1) / AT;
     float rc[ITEMS], rs[ITEMS];
 #pragma unroll
     for (int e = 0; e < ITEMS; ++e) {
         const int i = tid + e * AT;
         rc[e] = 1.f; rs[e] = 0.f;
         if (i < m * half && p.rope_cos) {
-            const size_t at = (size_t)(p.n_old + (p.tree ? (int)p.tdepth[i / half] : i / half)) * half + i % half;
+            const size_t at = (size_t)(n_old + (p.tree ? (int)p.tdepth[i / half] : i / half)) * half + i % half;
             rc[e] = p.rope_cos[at]; rs[e] = p.rope_sin[at];
         }
     }
@@ -480,7 +486,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
             const int i = tid + e * AT;
             if (i < m * half) {
                 const int r = i / half, d = i % half;
-                const float* qr = p.q + (size_t)r * p.ldq + h * DH;
+                const float* qr = p.q + (size_t)(r0 + r) * p.ldq + h * DH;
                 qv[e][0] = qr[d]; qv[e][1] = qr[d + half];
                 if (p.k_new) {
                     const float* kr = p.k_new + (size_t)r * p.ld_new + h * DH;
@@ -494,7 +500,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
         for (int e = 0; e < ITEMS; ++e) {
             const int i = tid + e * AT;
             if (i < m * half) {
-                const int r = i / half, d = i % half, pos = p.n_old + r;
+                const int r = i / half, d = i % half, pos = n_old + r;
                 const float c = rc[e], s = rs[e];
                 __nv_bfloat16 h0, l0, h1, l1;
                 split2(qv[e][0] * c - qv[e][1] * s, h0, l0);
@@ -540,9 +546,9 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
         unsigned char* Vt = Vs + st * C::TILE_BYTES;
         const int valid = min(TILE, s_end - t0);
         {
-            const int new_lo = max(t0, p.n_old), n_new = t0 + valid - new_lo;
+            const int new_lo = max(t0, n_old), n_new = t0 + valid - new_lo;
             for (int idx = tid; idx < n_new * (DH / 8); idx += AT) {
-                const int row = idx / (DH / 8), c = idx % (DH / 8), j = new_lo + row - t0, r = new_lo + row - p.n_old;
+                const int row = idx / (DH / 8), c = idx % (DH / 8), j = new_lo + row - t0, r = new_lo + row - n_old;
                 *reinterpret_cast<uint4*>(Kt + kv_off<DH>(j, c)) = *reinterpret_cast<const uint4*>(newK + r * DH + c * 8);
                 *reinterpret_cast<uint4*>(Vt + kv_off<DH>(j, c)) = *reinterpret_cast<const uint4*>(newV + r * DH + c * 8);
             }
@@ -584,14 +590,14 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                 for (int e = 0; e < 4; ++e) {
                     const int r = mt * 16 + (lane >> 2) + (e >> 1) * 8, j = 8 * warp + (lane & 3) * 2 + (e & 1);
                     if (r < m) {
-                        const int key = t0 + j, limit = p.causal ? p.n_keys + r : p.n_keys;
+                        const int key = t0 + j, limit = p.causal ? n_keys + r : n_keys;
                         float s = -INFINITY;
                         bool vis = key < s_end && key < limit;
-                        if (p.tree && key >= p.n_old) vis = key < s_end && ((p.tmask[r] >> (key - p.n_old)) & 1u);
+                        if (p.tree && key >= n_old) vis = key < s_end && ((p.tmask[r] >> (key - n_old)) & 1u);
                         if (vis) {
                             s = sacc[mt][e] * p.scale;
                             if (bias_h) {
-                                int bi = key - (p.q_pos0 + r) + p.bias_zero;
+                                int bi = key - (p.q_pos0 + r0 + r) + p.bias_zero;
                                 bi = max(0, min(p.bias_len - 1, bi));
                                 s += bias_h[bi];
                             }
@@ -676,9 +682,9 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
 #pragma unroll
                     for (int t = 0; t < 2; ++t) {
                         const int d = 16 * warp + 8 * t + 2 * (lane & 3);
-                        float* dst = p.out + (size_t)r * p.ldo + h * DH + d;
+                        float* dst = p.out + (size_t)(r0 + r) * p.ldo + h * DH + d;
                         dst[0] = o[mt][t][2 * hr] * inv; dst[1] = o[mt][t][2 * hr + 1] * inv;
-                        if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, p.xs_m, p.xs_r0 + r, h * DH + d, dst[0], dst[1]);
+                        if (p.out_xs) store_split(p.out_xs, p.out_xs_ld, p.xs_m, p.xs_r0 + r0 + r, h * DH + d, dst[0], dst[1]);
                     }
                 }
         }
@@ -702,7 +708,7 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     }
     if (tid < m) { rec[tid * C::REC + DH] = row_m[tid]; rec[tid * C::REC + DH + 1] = row_l[tid]; }
     cluster.sync();
-    merge_splits<DH, C::REC>(cluster, rec, p, h, split);
+    merge_splits<DH, C::REC>(cluster, rec, p, h, split, m, r0);
     cluster.sync();       // no CTA leaves while another may still read its record
 }
 // One 64-key tile per CTA while that keeps the splits of a head inside one portable cluster (8)
@@ -723,7 +729,8 @@ int attn_splits(int total_keys, int H) {
 static void attn_launch_config(cudaLaunchConfig_t& cfg, cudaLaunchAttribute* attr, const AttnParams& ap, size_t smem,
                                cudaStream_t st) {
     cfg = cudaLaunchConfig_t{};
-    cfg.gridDim = dim3((unsigned)ap.H, (unsigned)ap.nsplit);
+    cfg.gridDim = dim3((unsigned)ap.H, (unsigned)ap.nsplit,
+                       (unsigned)(ap.sub_rows > 0 ? (ap.m + ap.sub_rows - 1) / ap.sub_rows : 1));
     cfg.blockDim = dim3(AT);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = st;
@@ -768,8 +775,34 @@ static csd_status launch_mma(const CUtensorMap& tk, const CUtensorMap& tv, const
     return CSD_OK;
 }
 
+// Blocks of more than MAXM rows over a cache that already holds their keys (wide prefill, encoder):
+// one launch whose grid.z walks sub-blocks of 32 rows on the tensor-core kernel; elsewhere one
+// launch per MAXM rows.
+static csd_status launch_attention_rows(const AttnArgs& a, cudaStream_t st);
+static csd_status launch_attention_block(const AttnArgs& a, int sub_rows, cudaStream_t st);
+
 csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
-    if (!a.q || !a.Kc || !a.Vc || !a.out || a.m < 1 || a.m > MAXM || a.H < 1 || a.n_keys < 0)
+    if (a.m > MAXM) return launch_attention_rows(a, st);
+    return launch_attention_block(a, 0, st);
+}
+
+static csd_status launch_attention_rows(const AttnArgs& a, cudaStream_t st) {
+    if (a.k_new || a.tree_mask || a.out_xs || a.m > 128) return CSD_ERR_INVALID_ARG;   // 128: the widest block the model driver forms
+    if ((a.Dh == 64 || a.Dh == 128) && !g_attn_cuda_cores) return launch_attention_block(a, 32, st);
+    for (int r0 = 0; r0 < a.m; r0 += MAXM) {
+        AttnArgs s = a;
+        s.q = a.q + (size_t)r0 * a.ldq; s.m = a.m - r0 < MAXM ? a.m - r0 : MAXM;
+        s.n_keys = a.causal ? a.n_keys + r0 : a.n_keys;
+        s.q_pos0 = a.q_pos0 + r0;
+        s.out = a.out + (size_t)r0 * a.ldo;
+        const csd_status rc = launch_attention_block(s, 0, st);
+        if (rc != CSD_OK) return rc;
+    }
+    return CSD_OK;
+}
+
+static csd_status launch_attention_block(const AttnArgs& a, int sub_rows, cudaStream_t st) {
+    if (!a.q || !a.Kc || !a.Vc || !a.out || a.m < 1 || (sub_rows == 0 && a.m > MAXM) || a.H < 1 || a.n_keys < 0)
         return CSD_ERR_INVALID_ARG;
     const bool append = a.k_new != nullptr;
     if (append && (!a.v_new || !a.causal || a.n_keys < 1)) return CSD_ERR_INVALID_ARG;
@@ -793,7 +826,10 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
         ap.tree = 1;
         for (int r = 0; r < MAXM; ++r) { ap.tmask[r] = r < a.m ? a.tree_mask[r] : 0u; ap.tdepth[r] = r < a.m ? (unsigned char)a.tree_depth[r] : 0; }
     }
-    ap.nsplit = attn_splits(total, a.H);
+    ap.sub_rows = sub_rows;
+    // sub-blocks: each (head, sub-block) pair is a cluster of its own; the split length follows the
+    // last sub-block, which sees the most keys (earlier ones leave their last splits empty)
+    ap.nsplit = attn_splits(total, sub_rows > 0 ? a.H * ((a.m + sub_rows - 1) / sub_rows) : a.H);
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;
     ap.nsplit = (total + ap.split_len - 1) / ap.split_len;
@@ -801,10 +837,12 @@ csd_status launch_attention(const AttnArgs& a, cudaStream_t st) {
     if ((a.Dh == 64 || a.Dh == 128) && !g_attn_cuda_cores) {
         CUtensorMap tk, tv;
         if (tensor_map_2d(a.Kc, a.H * a.cap, a.Dh, TILE, &tk) && tensor_map_2d(a.Vc, a.H * a.cap, a.Dh, TILE, &tv)) {
-            if (a.Dh == 64) return a.m <= 16 ? launch_mma<64, 1>(tk, tv, ap, st) : launch_mma<64, 2>(tk, tv, ap, st);
-            return a.m <= 16 ? launch_mma<128, 1>(tk, tv, ap, st) : launch_mma<128, 2>(tk, tv, ap, st);
+            const bool one_tile = sub_rows == 0 && a.m <= 16;
+            if (a.Dh == 64) return one_tile ? launch_mma<64, 1>(tk, tv, ap, st) : launch_mma<64, 2>(tk, tv, ap, st);
+            return one_tile ? launch_mma<128, 1>(tk, tv, ap, st) : launch_mma<128, 2>(tk, tv, ap, st);
         }
     }
+    if (sub_rows > 0) return CSD_ERR_UNSUPPORTED;     // sub-blocks exist on the tensor-core kernel only
     switch (a.Dh) {
         case 32: return launch_dh<32>(ap, st);
         case 64: return launch_dh<64>(ap, st);

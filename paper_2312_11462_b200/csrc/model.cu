@@ -318,23 +318,20 @@ static csd_status wide_linear(csd_model* M, const __nv_bfloat16* W, const __nv_b
     return launch_linear_wide(a, st);
 }
 
-// Attention of `m` rows (any number) in sub-blocks of at most CSD_MAX_ROWS over K/V that are already
-// in the cache: row r sees keys [0, n_keys0 + r) when causal, all n_keys0 otherwise.
+// Attention of `m` <= CSD_WIDE_ROWS rows over K/V that are already in the cache: row r sees keys
+// [0, n_keys0 + r) when causal, all n_keys0 otherwise.
 static csd_status wide_attention(csd_model* M, const float* q, int ldq, int m, __nv_bfloat16* Kc, __nv_bfloat16* Vc, int cap,
                                  int n_keys0, bool causal, const float* bias, int bias_len, int bias_zero, int q_pos0,
                                  float* out, cudaStream_t st) {
     const csd_model_config& c = M->cfg;
-    for (int r0 = 0; r0 < m; r0 += CSD_MAX_ROWS) {
-        AttnArgs a;
-        a.q = q + (size_t)r0 * ldq; a.ldq = ldq; a.m = m - r0 < CSD_MAX_ROWS ? m - r0 : CSD_MAX_ROWS;
-        a.Kc = Kc; a.Vc = Vc; a.cap = cap; a.H = c.n_heads; a.Dh = c.d_head;
-        a.n_keys = causal ? n_keys0 + r0 : n_keys0; a.causal = causal ? 1 : 0;
-        a.scale = c.arch == 0 ? 1.f / sqrtf((float)c.d_head) : 1.f;
-        a.bias = bias; a.bias_len = bias_len; a.bias_zero = bias_zero; a.q_pos0 = q_pos0 + r0;
-        a.out = out + (size_t)r0 * M->di; a.ldo = M->di;
-        CSD_TRY(attention(M, a, st));
-    }
-    return CSD_OK;
+    AttnArgs a;       // one launch over all rows where the tensor-core kernel applies (sub-blocks in its grid)
+    a.q = q; a.ldq = ldq; a.m = m;
+    a.Kc = Kc; a.Vc = Vc; a.cap = cap; a.H = c.n_heads; a.Dh = c.d_head;
+    a.n_keys = n_keys0; a.causal = causal ? 1 : 0;
+    a.scale = c.arch == 0 ? 1.f / sqrtf((float)c.d_head) : 1.f;
+    a.bias = bias; a.bias_len = bias_len; a.bias_zero = bias_zero; a.q_pos0 = q_pos0;
+    a.out = out; a.ldo = M->di;
+    return attention(M, a, st);
 }
 
 // Decoder pass over m <= CSD_WIDE_ROWS rows at positions kv_len .. kv_len+m-1: K/V of every layer are
