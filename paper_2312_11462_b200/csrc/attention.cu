@@ -533,6 +533,25 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
     const int lrow = lane & 7, lmat = lane >> 3;          // ldmatrix: this lane addresses row lrow of matrix lmat
     const uint32_t qh_s = smem_u32(qh), ql_s = smem_u32(ql), ph_s = smem_u32(ph), pl_s = smem_u32(pl);
 
+    // The q operand is the same for every tile: each warp keeps the A fragments of its row tile in
+    // registers (high parts; the low parts too while a block is one row tile) instead of fetching
+    // them from shared memory per tile, which is what bounded the score step.  A warp takes the row
+    // tile mtw and MT groups of 8 keys of every tile.
+    constexpr bool QLO_REG = MT == 1;
+    const int mtw = MT == 1 ? 0 : warp >> 2;
+    const int key0 = MT == 1 ? 8 * warp : 16 * (warp & 3);
+    uint32_t qfh[DH / 16][4], qfl[QLO_REG ? DH / 16 : 1][4];
+    __syncthreads();                        // the block's q rows are in shared memory
+#pragma unroll
+    for (int ks = 0; ks < DH / 16; ++ks) {
+        const uint32_t aoff = (uint32_t)((mtw * 16 + (lmat & 1) * 8 + lrow) * C::QP + (2 * ks + (lmat >> 1)) * 16);
+        ldsm_x4(qh_s + aoff, qfh[ks]);
+        if (QLO_REG) ldsm_x4(ql_s + aoff, qfl[QLO_REG ? ks : 0]);
+    }
+
+    float run_m[R / 8], run_l[R / 8];       // running maximum and this lane's share of the running sum, rows warp + 8 i
+#pragma unroll
+    for (int i = 0; i < R / 8; ++i) { run_m[i] = -INFINITY; run_l[i] = 0.f; }
     bool failed = false;
     for (int it = 0; it < n_tiles; ++it) {
         const int st = it % STAGES, t0 = s_begin + it * TILE;
@@ -542,11 +561,16 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
             failed = true;
             break;
         }
+        // every thread is past the previous tile (the barrier above): its stage may be filled again
+        if (tid == 0 && it >= 1 && it - 1 + STAGES < n_tiles) {
+            fence_async_smem();
+            request(it - 1 + STAGES);
+        }
         unsigned char* Kt = Ks + st * C::TILE_BYTES;
         unsigned char* Vt = Vs + st * C::TILE_BYTES;
         const int valid = min(TILE, s_end - t0);
-        {
-            const int new_lo = max(t0, n_old), n_new = t0 + valid - new_lo;
+        const int new_lo = max(t0, n_old), n_new = t0 + valid - new_lo;
+        if (n_new > 0 || valid < TILE) {       // same for every thread
             for (int idx = tid; idx < n_new * (DH / 8); idx += AT) {
                 const int row = idx / (DH / 8), c = idx % (DH / 8), j = new_lo + row - t0, r = new_lo + row - n_old;
                 *reinterpret_cast<uint4*>(Kt + kv_off<DH>(j, c)) = *reinterpret_cast<const uint4*>(newK + r * DH + c * 8);
@@ -556,46 +580,51 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                 const int j = valid + idx / (DH / 8), c = idx % (DH / 8);
                 *reinterpret_cast<uint4*>(Vt + kv_off<DH>(j, c)) = make_uint4(0, 0, 0, 0);
             }
+            __syncthreads();
         }
-        __syncthreads();
-        // ---- scores of keys 8*warp .. 8*warp+7 for all rows
+        // ---- scores of this warp's row tile against its MT groups of 8 keys; the high and low parts of q and
+        //      the two halves of the head dimension accumulate separately, so that no chain is longer than DH/32 MMAs
         {
-            float sacc[MT][4];
+            float sacc2[MT][2][2][4];           // [key group][q part][half of the k steps]
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
+            for (int g = 0; g < MT; ++g)
 #pragma unroll
-                for (int e = 0; e < 4; ++e) sacc[mt][e] = 0.f;
+                for (int e = 0; e < 4; ++e)
+                    sacc2[g][0][0][e] = sacc2[g][0][1][e] = sacc2[g][1][0][e] = sacc2[g][1][1][e] = 0.f;
             const uint32_t Kt_s = smem_u32(Kt);
 #pragma unroll
             for (int ks2 = 0; ks2 < DH / 32; ++ks2) {
-                uint32_t kb[4];
-                ldsm_x4(Kt_s + kv_off<DH>(8 * warp + lrow, 4 * ks2 + lmat), kb);
 #pragma unroll
-                for (int hf = 0; hf < 2; ++hf) {
-                    const int ks = 2 * ks2 + hf;
+                for (int g = 0; g < MT; ++g) {
+                    uint32_t kb[4];
+                    ldsm_x4(Kt_s + kv_off<DH>(key0 + 8 * g + lrow, 4 * ks2 + lmat), kb);
 #pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        const uint32_t aoff = (uint32_t)((mt * 16 + (lmat & 1) * 8 + lrow) * C::QP + (2 * ks + (lmat >> 1)) * 16);
-                        uint32_t a[4];
-                        ldsm_x4(qh_s + aoff, a);
-                        mma_bf16(sacc[mt], a, kb[2 * hf], kb[2 * hf + 1]);
-                        ldsm_x4(ql_s + aoff, a);
-                        mma_bf16(sacc[mt], a, kb[2 * hf], kb[2 * hf + 1]);
+                    for (int hf = 0; hf < 2; ++hf) {
+                        const int ks = 2 * ks2 + hf;
+                        mma_bf16(sacc2[g][0][hf], qfh[ks], kb[2 * hf], kb[2 * hf + 1]);
+                        if (QLO_REG) {
+                            mma_bf16(sacc2[g][1][hf], qfl[QLO_REG ? ks : 0], kb[2 * hf], kb[2 * hf + 1]);
+                        } else {
+                            const uint32_t aoff = (uint32_t)((mtw * 16 + (lmat & 1) * 8 + lrow) * C::QP + (2 * ks + (lmat >> 1)) * 16);
+                            uint32_t a[4];
+                            ldsm_x4(ql_s + aoff, a);
+                            mma_bf16(sacc2[g][1][hf], a, kb[2 * hf], kb[2 * hf + 1]);
+                        }
                     }
                 }
             }
 #pragma unroll
-            for (int mt = 0; mt < MT; ++mt)
+            for (int g = 0; g < MT; ++g)
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const int r = mt * 16 + (lane >> 2) + (e >> 1) * 8, j = 8 * warp + (lane & 3) * 2 + (e & 1);
+                    const int r = mtw * 16 + (lane >> 2) + (e >> 1) * 8, j = key0 + 8 * g + (lane & 3) * 2 + (e & 1);
                     if (r < m) {
                         const int key = t0 + j, limit = p.causal ? n_keys + r : n_keys;
                         float s = -INFINITY;
                         bool vis = key < s_end && key < limit;
                         if (p.tree && key >= n_old) vis = key < s_end && ((p.tmask[r] >> (key - n_old)) & 1u);
                         if (vis) {
-                            s = sacc[mt][e] * p.scale;
+                            s = ((sacc2[g][1][0][e] + sacc2[g][1][1][e]) + (sacc2[g][0][0][e] + sacc2[g][0][1][e])) * p.scale;
                             if (bias_h) {
                                 int bi = key - (p.q_pos0 + r0 + r) + p.bias_zero;
                                 bi = max(0, min(p.bias_len - 1, bi));
@@ -607,30 +636,44 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                 }
         }
         __syncthreads();
-        // ---- online softmax: warp w owns rows w, w+8, w+16; the weights leave as bf16 pairs
-        for (int r = warp; r < m; r += AT / 32) {
-            const float s0 = sc[r * C::SP + lane], s1 = sc[r * C::SP + lane + 32];
-            const float tmax = warp_max(fmaxf(s0, s1));
-            const float old = row_m[r];
-            const float nm = fmaxf(old, tmax);
-            float p0 = 0.f, p1 = 0.f, alpha = 1.f;
-            if (nm > -INFINITY) {
-                p0 = expf(s0 - nm);
-                p1 = expf(s1 - nm);
-                alpha = expf(old - nm);
+        // ---- online softmax: warp w owns rows w, w+8, ...; the weights leave as bf16 pairs.  The rows of a
+        //      warp are independent, so their loads, shuffles and exponentials interleave; the row sums stay
+        //      as per-lane partial sums until the walk is over.
+        {
+            float s0[R / 8], s1[R / 8], tmax[R / 8];
+#pragma unroll
+            for (int i = 0; i < R / 8; ++i) {
+                const int r = warp + 8 * i;
+                s0[i] = s1[i] = -INFINITY;
+                if (r < m) { s0[i] = sc[r * C::SP + lane]; s1[i] = sc[r * C::SP + lane + 32]; }
+                tmax[i] = fmaxf(s0[i], s1[i]);
             }
-            __nv_bfloat16 h0, l0, h1, l1;
-            split2(p0, h0, l0);
-            split2(p1, h1, l1);
-            __nv_bfloat16* phr = reinterpret_cast<__nv_bfloat16*>(ph + r * C::PP);
-            __nv_bfloat16* plr = reinterpret_cast<__nv_bfloat16*>(pl + r * C::PP);
-            phr[lane] = h0; phr[lane + 32] = h1; plr[lane] = l0; plr[lane + 32] = l1;
-            // the sum runs over the weights as the MMA will see them
-            const float tsum = warp_sum((__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1)));
-            if (lane == 0) {
-                row_m[r] = nm;
-                row_l[r] = row_l[r] * alpha + tsum;
-                row_a[r] = alpha;
+#pragma unroll
+            for (int off = 16; off > 0; off >>= 1)
+#pragma unroll
+                for (int i = 0; i < R / 8; ++i) tmax[i] = fmaxf(tmax[i], __shfl_xor_sync(0xffffffffu, tmax[i], off));
+#pragma unroll
+            for (int i = 0; i < R / 8; ++i) {
+                const int r = warp + 8 * i;
+                if (r >= m) continue;
+                const float old = run_m[i];
+                const float nm = fmaxf(old, tmax[i]);
+                float p0 = 0.f, p1 = 0.f, alpha = 1.f;
+                if (nm > -INFINITY) {
+                    p0 = expf(s0[i] - nm);
+                    p1 = expf(s1[i] - nm);
+                    alpha = expf(old - nm);
+                }
+                __nv_bfloat16 h0, l0, h1, l1;
+                split2(p0, h0, l0);
+                split2(p1, h1, l1);
+                __nv_bfloat16* phr = reinterpret_cast<__nv_bfloat16*>(ph + r * C::PP);
+                __nv_bfloat16* plr = reinterpret_cast<__nv_bfloat16*>(pl + r * C::PP);
+                phr[lane] = h0; phr[lane + 32] = h1; plr[lane] = l0; plr[lane + 32] = l1;
+                // the sum runs over the weights as the MMA will see them
+                run_l[i] = run_l[i] * alpha + ((__bfloat162float(h0) + __bfloat162float(l0)) + (__bfloat162float(h1) + __bfloat162float(l1)));
+                run_m[i] = nm;
+                if (lane == 0) row_a[r] = alpha;
             }
         }
         __syncthreads();
@@ -643,6 +686,13 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                 for (int t = 0; t < 2; ++t) { o[mt][t][0] *= a0; o[mt][t][1] *= a0; o[mt][t][2] *= a1; o[mt][t][3] *= a1; }
             }
             const uint32_t Vt_s = smem_u32(Vt);
+            float ol[MT][2][4];                 // the low parts of the weights accumulate on their own chain
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) ol[mt][t][e] = 0.f;
 #pragma unroll
             for (int ks = 0; ks < TILE / 16; ++ks) {
                 uint32_t vb[4];
@@ -655,18 +705,26 @@ block_attention_mma_kernel(const __grid_constant__ CUtensorMap tmK, const __grid
                     mma_bf16(o[mt][0], a, vb[0], vb[1]);
                     mma_bf16(o[mt][1], a, vb[2], vb[3]);
                     ldsm_x4(pl_s + aoff, a);
-                    mma_bf16(o[mt][0], a, vb[0], vb[1]);
-                    mma_bf16(o[mt][1], a, vb[2], vb[3]);
+                    mma_bf16(ol[mt][0], a, vb[0], vb[1]);
+                    mma_bf16(ol[mt][1], a, vb[2], vb[3]);
                 }
             }
-        }
-        __syncthreads();           // tile consumed: its stage may be filled again
-        if (tid == 0 && it + STAGES < n_tiles) {
-            fence_async_smem();
-            request(it + STAGES);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int t = 0; t < 2; ++t)
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) o[mt][t][e] += ol[mt][t][e];
         }
     }
     if (failed && tid == 0) set_status(p.status, CSD_ERR_TIMEOUT);
+#pragma unroll
+    for (int i = 0; i < R / 8; ++i) {
+        const float l = warp_sum(run_l[i]);
+        const int r = warp + 8 * i;
+        if (lane == 0 && r < m) { row_m[r] = run_m[i]; row_l[r] = l; }
+    }
+    __syncthreads();
 
 
     // element (mt, t, e) of `o`: row mt*16 + lane/4 (+8 for e >= 2), dimension 16*warp + 8*t + 2*(lane%4) + (e&1)
