@@ -320,11 +320,13 @@ resample_z_kernel(const float* __restrict__ tl, const float* __restrict__ dl, in
                   const RowInfo* __restrict__ info, double2* __restrict__ zpart, double2* __restrict__ zsum,
                   unsigned* __restrict__ tickets, int nchunk) {
     const int row = blockIdx.x, chunk = blockIdx.y;
-    const RowInfo ri = info[row];
-    if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
     __shared__ double s_tab[64];
     exp_table_to_shared(s_tab);
+    pdl_wait();            // the row records come from the decide pass
+    pdl_trigger();
+    const RowInfo ri = info[row];
+    if (ri.mode == MODE_DONE) return;
     const double invT = 1.0 / (double)temperature;
     const float* t = tl + ((long long)row * (k + 1) + ri.n) * V;
     const float* d = ri.mode == MODE_RESID_LOGITS ? dl + ((long long)row * k + ri.n) * V : nullptr;
@@ -375,6 +377,8 @@ resample_pick_kernel(const float* __restrict__ tl, const float* __restrict__ dl,
                      const double2* __restrict__ zsum, double* __restrict__ rpart, unsigned* __restrict__ tickets,
                      int nchunk, int* __restrict__ out_tok) {
     const int row = blockIdx.x, chunk = blockIdx.y;
+    pdl_wait();            // the normalisers come from the pass before this one
+    pdl_trigger();
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;
     __shared__ double s_warp[RS_THREADS / 32];
@@ -551,6 +555,8 @@ resample_fused_kernel(const float* __restrict__ tl, const float* __restrict__ dl
                       const RowInfo* __restrict__ info, int csize, int* __restrict__ out_tok) {
     const int row = blockIdx.x / csize;
     const uint32_t rank = cluster_rank();
+    pdl_wait();            // the row records come from the decide pass
+    pdl_trigger();
     const RowInfo ri = info[row];
     if (ri.mode == MODE_DONE) return;                 // (the same decision in every CTA of the cluster)
     __shared__ double s_warp[RF_THREADS / 32];
@@ -791,18 +797,24 @@ static csd_status run_accept(const float* tl, const float* dl_in, const int32_t*
     }
     if (!greedy && fused_resample_ok(csize)) {  // a row fits one cluster: the fused resample kernel
         cudaLaunchConfig_t cfg = cudaLaunchConfig_t{};
-        cudaLaunchAttribute attr[1];
+        cudaLaunchAttribute attr[2];
         cfg.gridDim = dim3((unsigned)(rows * csize)); cfg.blockDim = dim3(RF_THREADS); cfg.dynamicSmemBytes = 0; cfg.stream = st;
         attr[0].id = cudaLaunchAttributeClusterDimension;
         attr[0].val.clusterDim.x = (unsigned)csize; attr[0].val.clusterDim.y = 1; attr[0].val.clusterDim.z = 1;
-        cfg.attrs = attr; cfg.numAttrs = 1;
+        attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[1].val.programmaticStreamSerializationAllowed = 1;
+        cfg.attrs = attr; cfg.numAttrs = 2;
         CSD_CUDA(cudaLaunchKernelEx(&cfg, resample_fused_kernel, tl, dl, k, V, temperature, (const RowInfo*)info, csize,
                                     (int*)out_tok));
         count_launch();
     } else if (!greedy) {
         dim3 g2((unsigned)rows, (unsigned)L.nchunk_r);
-        resample_z_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, tickets, L.nchunk_r);
-        resample_pick_kernel<<<g2, RS_THREADS, 0, st>>>(tl, dl, k, V, temperature, info, zpart, zsum, rpart, tickets + rows, L.nchunk_r, out_tok);
+        PdlLaunch lz(g2, dim3(RS_THREADS), 0, st);
+        CSD_CUDA(cudaLaunchKernelEx(&lz.cfg, resample_z_kernel, tl, dl, k, V, temperature, (const RowInfo*)info, zpart, zsum, tickets,
+                                    L.nchunk_r));
+        PdlLaunch lp(g2, dim3(RS_THREADS), 0, st);
+        CSD_CUDA(cudaLaunchKernelEx(&lp.cfg, resample_pick_kernel, tl, dl, k, V, temperature, (const RowInfo*)info,
+                                    (const double2*)zpart, (const double2*)zsum, rpart, tickets + rows, L.nchunk_r, (int*)out_tok));
         count_launch(2);
     }
     CSD_CUDA(cudaGetLastError());
