@@ -26,6 +26,53 @@ __global__ void embed_kernel(const int32_t* __restrict__ tokens, const __nv_bflo
     for (int i = threadIdx.x; i < d; i += blockDim.x) x[(size_t)r * d + i] = __bfloat162float(e[i]);
 }
 
+// The same gather for a forward whose first projection runs on the tensor cores: besides the fp32 rows it
+// writes the rows times `gain` as three bf16 terms (rows term * m + r of xs) and the pieces of each row's sum
+// of squares, i.e. what the stand-alone split of those rows would write next.  grid = (d / 1024 rounded up, m).
+__global__ void __launch_bounds__(128)
+embed_split_kernel(const int32_t* __restrict__ tokens, const __nv_bfloat16* __restrict__ E, int V, int d, int m,
+                   const __nv_bfloat16* __restrict__ gain, float* __restrict__ x, __nv_bfloat16* __restrict__ xs,
+                   float* __restrict__ ssq, int* status) {
+    pdl_wait();
+    pdl_trigger();
+    const int r = blockIdx.y, k = (blockIdx.x * 128 + threadIdx.x) * 8;
+    int t = tokens[r];
+    if (t < 0 || t >= V) {
+        if (threadIdx.x == 0 && blockIdx.x == 0) set_status(status, CSD_ERR_BAD_TOKEN);
+        t = 0;
+    }
+    float sq = 0.f;
+    if (k < d) {
+        const uint4 e = *reinterpret_cast<const uint4*>(E + (size_t)t * d + k);
+        float v[8] = {bf16lo(e.x), bf16hi(e.x), bf16lo(e.y), bf16hi(e.y), bf16lo(e.z), bf16hi(e.z), bf16lo(e.w), bf16hi(e.w)};
+        float* dst = x + (size_t)r * d + k;
+        *reinterpret_cast<float4*>(dst) = make_float4(v[0], v[1], v[2], v[3]);
+        *reinterpret_cast<float4*>(dst + 4) = make_float4(v[4], v[5], v[6], v[7]);
+#pragma unroll
+        for (int i = 0; i < 8; ++i) sq = fmaf(v[i], v[i], sq);
+        const uint4 g = *reinterpret_cast<const uint4*>(gain + k);
+        v[0] *= bf16lo(g.x); v[1] *= bf16hi(g.x); v[2] *= bf16lo(g.y); v[3] *= bf16hi(g.y);
+        v[4] *= bf16lo(g.z); v[5] *= bf16hi(g.z); v[6] *= bf16lo(g.w); v[7] *= bf16hi(g.w);
+        uint32_t w[3][4];
+#pragma unroll
+        for (int i = 0; i < 8; i += 2) {
+            uint16_t a1, a2, a3, c1, c2, c3;
+            split3(v[i], a1, a2, a3);
+            split3(v[i + 1], c1, c2, c3);
+            w[0][i / 2] = a1 | ((uint32_t)c1 << 16); w[1][i / 2] = a2 | ((uint32_t)c2 << 16);
+            w[2][i / 2] = a3 | ((uint32_t)c3 << 16);
+        }
+#pragma unroll
+        for (int u = 0; u < 3; ++u)
+            *reinterpret_cast<uint4*>(xs + (size_t)(u * m + r) * d + k) = make_uint4(w[u][0], w[u][1], w[u][2], w[u][3]);
+    }
+    __shared__ float part[4];
+    sq = warp_sum(sq);
+    if ((threadIdx.x & 31) == 0) part[threadIdx.x >> 5] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) ssq[(size_t)blockIdx.x * m + r] = (part[0] + part[1]) + (part[2] + part[3]);
+}
+
 // cos/sin of pos * theta^(-2i/Dh), evaluated in double once per model
 __global__ void rope_table_kernel(float* __restrict__ cs, float* __restrict__ sn, int max_seq, int half, double theta) {
     const int idx = blockIdx.x * blockDim.x + threadIdx.x;
@@ -736,14 +783,24 @@ static csd_status review_forward_impl(csd_model* M, const int32_t* block_tokens_
     if (c.arch == 1 && M->enc_len < 1) return CSD_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     const int d = c.d_model, H = c.n_heads, Dh = c.d_head, di = M->di, V = c.vocab;
+    // x_ready: M->xs_x / M->ssq_x hold the residual rows (times the gain of the norm that reads them
+    // next) in three-term form, written by the epilogue of the GEMM that produced the rows (for the
+    // embedded rows: by the gather itself, when the first projection takes that form)
+    bool x_ready = false;
     {
         ProfScope ps(M, 2, st);
-        embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
+        const LayerW& y0 = M->dec[0];
+        const bool fused_qkv = y0.wk == y0.wq + (size_t)di * d && y0.wv == y0.wk + (size_t)di * d;
+        if ((d & 7) == 0 && linear_uses_tensor_cores(m, fused_qkv ? 3 * di : di, d, false)) {
+            embed_split_kernel<<<dim3((unsigned)split_ssq_entries(d), (unsigned)m), 128, 0, st>>>(
+                block_tokens_dev, M->embed, V, d, m, y0.norm1, M->x, M->xs_x, M->ssq_x, M->status);
+            M->ssq_x_cnt = split_ssq_entries(d);
+            x_ready = true;
+        } else {
+            embed_kernel<<<m, 128, 0, st>>>(block_tokens_dev, M->embed, V, d, M->x, M->status);
+        }
         count_launch();
     }
-    // x_ready: M->xs_x / M->ssq_x hold the residual rows (times the gain of the norm that reads them
-    // next) in three-term form, written by the epilogue of the GEMM that produced the rows
-    bool x_ready = false;
     const int ff = c.d_ff;
     const bool tc_o = linear_uses_tensor_cores(m, d, di, false);
     for (int l = 0; l < c.n_layers; ++l) {
