@@ -287,8 +287,9 @@ def run_ours(args):
     # a short sample of every other configuration, so that each has a figure in this line
     other = None
     if world == 1 and not args.no_configs:
+        variants = cfg_variants(b, ts, tb, target, prompt, draft, nxt_dev)
         draft.close()
-        other = {"variants": cfg_variants(b, ts, tb, target, prompt), "tiny_cascade": cfg_tiny(b),
+        other = {"variants": variants, "tiny_cascade": cfg_tiny(b),
                  "accept": [cfg_accept(b, peak, 128256, 16, 0.5), cfg_accept(b, peak, 128256, 4, 0.5),
                             cfg_accept(b, peak, 32000, 4, 0.5)],
                  "long_cache_review_step": cfg_long(b, peak, tb, reviews=6)}
@@ -472,7 +473,7 @@ def cfg_long(b, peak, tb, block_rows=(2, 5, 9, 17), reviews=8, S=2048):
     return out
 
 
-def cfg_variants(b, ts, tb, target, prompt):
+def cfg_variants(b, ts, tb, target, prompt, draft=None, nxt_dev=None):
     """Review-step variants on the 7B-shaped target: a tree-shaped block (the paper's tree-attention
     setting: eight candidates at the first position, the lead continued by a chain of three) and a
     batched review (three sequences of five rows in one pass over the weights)."""
@@ -499,8 +500,19 @@ def cfg_variants(b, ts, tb, target, prompt):
     batch_us = timed_us(lambda i: b.csd_review_forward_batch(models, blocks, [PROMPT_LEN] * 3), 10)
     for m_ in others:
         m_.close()
-    return {"tree_review_step": {"rows": len(parent), "shape": "8 candidates at the first position, lead + chain of 3", "us": tree_us},
-            "batched_review": {"sequences": 3, "rows_each": MAX_BLOCK + 1, "us": batch_us, "us_per_sequence": batch_us / 3}}
+    res = {"tree_review_step": {"rows": len(parent), "shape": "8 candidates at the first position, lead + chain of 3", "us": tree_us},
+           "batched_review": {"sequences": 3, "rows_each": MAX_BLOCK + 1, "us": batch_us, "us_per_sequence": batch_us / 3}}
+    if draft is not None:
+        # the same models under the paper's budget matrix for this pair (Appendix B: [[2,10],[0,10]]): the draft
+        # reviews ten Max-Gram tokens at a time, the target two draft tokens; blocks of up to 16 drafts
+        casc = b.Cascade([target, draft], [[2, 10], [0, 10]], 16, nxt_dev, PROMPT_LEN)
+        casc.csd_cascade_generate(prompt, prompt, 32)
+        toks, st = casc.csd_cascade_generate(prompt, prompt, MAX_NEW)
+        res["paper_budget_matrix"] = {"K": [[2, 10], [0, 10]], "max_block": 16, "new_tokens": len(toks),
+                                      "tokens_per_s": len(toks) / (1e-3 * (st["prefill_ms"] + st["decode_ms"])),
+                                      "target_forwards_per_token": st["forwards"][0] / max(len(toks), 1),
+                                      "reviews": st["reviews"], "accepted": st["accepted"], "mag_tokens": st["mag_tokens"]}
+    return res
 
 
 def cfg_t5(b, cascade=True):
