@@ -43,6 +43,14 @@ def test_layer_shapes(b, orc, m):
         case(b, orc, m, N, K, seed=N + K + m)
 
 
+def test_every_block_size(b, orc):
+    # all seventeen row counts (every operand padding of the tensor-core kernels: 16, 32, 48, 64 rows of
+    # terms) on a shape with several tiles per CTA share and on one with a single short tile
+    for m in range(1, 18):
+        case(b, orc, m, 3072, 4096, seed=100 + m)
+        case(b, orc, m, 200, 1160, seed=200 + m)
+
+
 @pytest.mark.parametrize("N,K", [(4096, 4096), (12288, 4096), (4096, 11008)])
 def test_7b_layer_shapes(b, orc, N, K):
     for m in (5, 17):
