@@ -888,6 +888,14 @@ static csd_status launch_attention_block(const AttnArgs& a, int sub_rows, cudaSt
     // sub-blocks: each (head, sub-block) pair is a cluster of its own; the split length follows the
     // last sub-block, which sees the most keys (earlier ones leave their last splits empty)
     ap.nsplit = attn_splits(total, sub_rows > 0 ? a.H * ((a.m + sub_rows - 1) / sub_rows) : a.H);
+    if (sub_rows > 0) {
+        // these launches are throughput-bound: as many splits as keep the whole grid resident at once
+        // (two CTAs per SM), rather than one more that spills into a second wave
+        const int pairs = a.H * ((a.m + sub_rows - 1) / sub_rows);
+        int fit = 2 * 148 / pairs;
+        if (fit < 1) fit = 1;
+        if (ap.nsplit > fit) ap.nsplit = fit;
+    }
     int len = (total + ap.nsplit - 1) / ap.nsplit;
     ap.split_len = (len + TILE - 1) / TILE * TILE;
     ap.nsplit = (total + ap.split_len - 1) / ap.split_len;
