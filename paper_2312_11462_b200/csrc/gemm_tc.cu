@@ -216,7 +216,12 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                       const __grid_constant__ CUtensorMap tmX, const TcParams p) {
     constexpr int NPAD = 3 * M <= 16 ? 16 : (3 * M <= 32 ? 32 : (3 * M <= 48 ? 48 : 64));
     constexpr int NT = DUAL ? 2 : 1;
-    constexpr int ACC_COLS = NPAD * NT;                       // tensor-memory columns per accumulator set
+    constexpr int ACC_ONE = NPAD * NT;                        // tensor-memory columns of one accumulator
+    // The tensor core's fp32 accumulation loses a little with every add of a long chain, so the K blocks
+    // of a segment go round-robin to NACC accumulators (as many as fit 256 columns twice over, at most
+    // 4); the epilogue adds them.
+    constexpr int NACC = 2 * ACC_ONE * 4 <= 256 ? 4 : (2 * ACC_ONE * 2 <= 256 ? 2 : 1);
+    constexpr int ACC_COLS = ACC_ONE * NACC;                  // columns per accumulator set (one segment)
     constexpr int TMEM_COLS = 2 * ACC_COLS <= 32 ? 32 : (2 * ACC_COLS <= 64 ? 64 : (2 * ACC_COLS <= 128 ? 128 : 256));
     constexpr int XBYTES = NPAD * 128;                        // the rows' terms for one K block
     constexpr int KS = (!DUAL && NPAD <= 16) ? 2 : 1;         // K blocks per stage
@@ -323,8 +328,10 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
                 kb_begin = 0;                     // later segments start at a tile's first K block
                 if (!mbar_wait(&ctl->acc_empty[b], ((seg >> 1) & 1) ^ 1)) { *abort_flag = 1; break; }
                 tc_fence_after();
-                const uint32_t d0 = tmem + (uint32_t)(b * ACC_COLS);
+                const uint32_t dset = tmem + (uint32_t)(b * ACC_COLS);
                 for (int j = 0; j < seg_len; ++j, ++i) {
+                    const uint32_t d0 = dset + (uint32_t)((j % NACC) * ACC_ONE);
+                    const int first = j < NACC ? 0 : 1;       // an accumulator's first K block overwrites it
                     if (!mbar_wait(&ctl->full[s], ph)) { *abort_flag = 1; break; }
                     tc_fence_after();
                     const uint64_t ad = desc0 + (uint64_t)(((uint32_t)s * (uint32_t)STAGE) >> 4);
@@ -334,8 +341,8 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 #pragma unroll
                         for (int k = 0; k < KB / 16; ++k) {
                             const uint64_t bdk = bd + ((h * XBYTES) >> 4) + 2 * k;
-                            tc_mma(d0, ad + ((h * STAGE_BYTES) >> 4) + 2 * k, bdk, IDESC, (j | h | k) != 0);
-                            if (DUAL) tc_mma(d0 + NPAD, ad + (STAGE_BYTES >> 4) + 2 * k, bdk, IDESC, (j | k) != 0);
+                            tc_mma(d0, ad + ((h * STAGE_BYTES) >> 4) + 2 * k, bdk, IDESC, (first | h | k) != 0);
+                            if (DUAL) tc_mma(d0 + NPAD, ad + (STAGE_BYTES >> 4) + 2 * k, bdk, IDESC, (first | k) != 0);
                         }
                     tc_commit(&ctl->empty[s]);          // stage reusable once these MMAs have read it
                     if (++s == p.stages) { s = 0; ph ^= 1u; }
@@ -371,16 +378,20 @@ skinny_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmW, const __grid_cons
 #pragma unroll
                 for (int r = 0; r < M; ++r) { sums[u][r] = 0.f; second[r] = 0.f; third[r] = 0.f; }
 #pragma unroll
-                for (int c0 = 0; c0 < NPAD; c0 += 16) {
-                    if (c0 >= 3 * M) break;
-                    float v[16];
-                    tc_ld16(taddr + (uint32_t)(u * NPAD + c0), v);
+                for (int a = 0; a < NACC; ++a) {
+                    if (a >= seg_len) break;            // a short segment used fewer accumulators
 #pragma unroll
-                    for (int c = 0; c < 16; ++c) {
-                        const int col = c0 + c;
-                        if (col < M) sums[u][col] = v[c];
-                        else if (col < 2 * M) second[col - M] = v[c];
-                        else if (col < 3 * M) third[col - 2 * M] = v[c];
+                    for (int c0 = 0; c0 < NPAD; c0 += 16) {
+                        if (c0 >= 3 * M) break;
+                        float v[16];
+                        tc_ld16(taddr + (uint32_t)(a * ACC_ONE + u * NPAD + c0), v);
+#pragma unroll
+                        for (int c = 0; c < 16; ++c) {
+                            const int col = c0 + c;
+                            if (col < M) sums[u][col] += v[c];
+                            else if (col < 2 * M) second[col - M] += v[c];
+                            else if (col < 3 * M) third[col - 2 * M] += v[c];
+                        }
                     }
                 }
 #pragma unroll
